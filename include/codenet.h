@@ -73,7 +73,9 @@ typedef struct {
                            /* alone (needs r >= 2); NODECHECK: locate with the inner          */
                            /* checksums, fall back to SYNDROME when nothing is flagged;       */
                            /* OFF: no check at all (timing baseline for the cost of the       */
-                           /* redundant blocks alone; injected errors pass through);          */
+                           /* redundant blocks alone; injected errors pass through; the inner */
+                           /* checksums are not maintained, and neither are they in a layer    */
+                           /* without parity blocks that runs no node check);                  */
                            /* JOINT: as SYNDROME ("Decoding Algorithm", Appendix B: the       */
                            /* block-sparsest e with (H x I) e = syndrome), but supports of up */
                            /* to r - 1 nodes (at most 3) instead of t = r / 2: the errors are  */

@@ -149,7 +149,6 @@ int codenet_encode_layer(const codenet_layer_desc_t* d, const void* W_dev, coden
   L->desc.P_row = nullptr;
   L->desc.P_col = nullptr;
   L->batch_max = d->batch_max;
-  L->check_parity = 0;
   L->out_act = CODENET_ACT_IDENTITY;
   L->out_mask = nullptr;
   L->next_x = nullptr;
@@ -207,8 +206,8 @@ int codenet_encode_layer(const codenet_layer_desc_t* d, const void* W_dev, coden
     if ((e = dev_alloc(&ws.xsum, (size_t)g.Nn * g.nsc * Bm)) != cudaSuccess) break;
     if ((e = dev_alloc(&ws.Y, ws.y_elems)) != cudaSuccess) break;
     if ((e = dev_alloc(&ws.Yw, ws.yw_elems)) != cudaSuccess) break;
-    if ((e = dev_alloc(&ws.tc_flag, (size_t)1)) != cudaSuccess) break;
-    if ((e = cudaMemsetAsync(ws.tc_flag, 0, sizeof(int), st)) != cudaSuccess) break;
+    if ((e = dev_alloc(&ws.tc_flag, (size_t)4)) != cudaSuccess) break;
+    if ((e = cudaMemsetAsync(ws.tc_flag, 0, 4 * sizeof(int), st)) != cudaSuccess) break;
     if (Bm > 8) {
       if ((e = dev_alloc(&ws.chk, check_scratch_floats(g, (int)Bm))) != cudaSuccess) break;
     }
@@ -222,9 +221,10 @@ int codenet_encode_layer(const codenet_layer_desc_t* d, const void* W_dev, coden
     // the update sweep can also take the next feedforward products when its column strips tile the
     // block-columns exactly and x needs no padding
     L->next_ok = (g.ldb % backward_strip_elems(g.dtype) == 0) && g.ldb == g.b_c && g.n * g.b_c == g.n_in;
+    const size_t Bs = Bm < 8 ? Bm : 8;   // the streaming path serves batches up to 8
     if (L->next_ok) {
       const size_t strips = (size_t)g.n * g.ldb / backward_strip_elems(g.dtype);
-      if ((e = dev_alloc(&ws.Ynext, strips * g.Mbr * (Bm < 8 ? Bm : 8))) != cudaSuccess) break;
+      if ((e = dev_alloc(&ws.Ynext, strips * g.Mbr * Bs)) != cudaSuccess) break;
     }
     if ((e = dev_alloc(&ws.stats, (size_t)2)) != cudaSuccess) break;
     if ((e = dev_alloc(&ws.plan, (size_t)CODENET_MAX_NODES)) != cudaSuccess) break;

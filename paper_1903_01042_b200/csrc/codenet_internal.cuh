@@ -29,6 +29,13 @@ struct Geom {
   const float* Pc;  // n x r_col
 };
 
+// Inner checksums are kept valid only where something can read them: not with the checks switched off, and not in
+// a layer without any parity block that runs no node check.
+__host__ __device__ inline bool keeps_checksums(const Geom& g) {
+  return g.locate_mode != CODENET_LOCATE_OFF &&
+         (g.r_row > 0 || g.r_col > 0 || g.locate_mode == CODENET_LOCATE_NODECHECK);
+}
+
 struct FaultDev {
   uint32_t seed, layer, mode, p_q32;
   float sigma;
@@ -69,9 +76,10 @@ struct Workspace {
   void* tc_d;     // tensor-core operand copy of delta~: (B, M*b_r), or NULL
   void* tc_dT;    // transposed operand copies for the update: (M*b_r, B) and (ld, B), or NULL
   void* tc_xT;
-  int* tc_flag;   // set by a tensor-core kernel whose bounded wait ran out
+  int* tc_flag;   // [0] set by a tensor-core kernel whose bounded wait ran out; [1] which statistics buffer the
+                  // next check kernel works in (kept on the device, flipped by the kernel)
   float* chk;     // inner-check scratch for batches > 8 (check_scratch_floats), or NULL
-  CheckStats* stats;  // two buffers used alternately; each call clears the other one
+  CheckStats* stats;  // two buffers used alternately; each check clears the other one
   CwPlan* plan;       // one per codeword
   size_t y_elems, yw_elems;
 };
@@ -86,7 +94,6 @@ struct codenet_layer {
   int batch_max;
   int bwd_rows;   // R: rows per tile of the fused backward+update kernel
   int bwd_rt;     // RT = ceil(b_r / R)
-  mutable int check_parity;  // which statistics buffer the next check uses
   int next_ok;               // the layout allows taking the next feedforward products in the update sweep
   const float* next_x;       // input those products were taken for (NULL: none pending)
   int next_B;

@@ -24,358 +24,15 @@
 
 #include <cooperative_groups.h>
 #include <float.h>
+#include <string.h>
 
 namespace cg = cooperative_groups;
 
 namespace codenet {
 namespace {
 
-constexpr int CK_THREADS = 256;
-constexpr int CK_WARPS = CK_THREADS / 32;
-constexpr int MAXR = CODENET_MAX_PARITY;
-constexpr int MAXN = CODENET_MAX_NODES;
-constexpr int BIG_WC = 8;     // large batches: 16-byte accesses in flight per lane
-constexpr int BIG_SR = 64;    // large batches: rows per work item of the statistics pass
-constexpr int BIG_DC = 128;   // large batches: dot-product entries per work item
-constexpr int BIG_TR = 16;    // large batches: positions per tile of the syndrome / sums pass
-constexpr int BIG_KD = 16;    // large batches: most data nodes per codeword the one-pass sums handle
+#include "check_device.cuh"
 
-struct CheckParams {
-  Geom g;
-  int phase, B, src_kind, have_clean, RT, commit, update_checksums, spb;  // spb: strips per block-column
-  float lr;
-  FaultDev fault;
-  const float* src;    // clean node outputs: canonical, or backward partials [i][rt][b][ld]
-  float* Yw;           // working copy [codeword][node][len][B]
-  const float* Vraw;   // X (B, n_in) for the forward check, Delta (B, n_out) for the backward check
-  float* out;          // S (B, n_out) / C (B, n_in) or NULL
-  const float* Xt; const float* Dt; const float* dsum; const float* xsum;
-  CheckStats* st; CheckStats* st_next;
-  CwPlan* plan;
-  codenet_report_t* rep;
-  const int* tc_flag;  // non-zero: a tensor-core kernel of this layer gave up on a bounded wait
-  float* chk;          // large batches: [unit][b][partials] of slice sum / magnitudes and checksum dot / scale
-  int lazy;                // large-batch path: node outputs stay where the product kernel wrote them, only
-                           // hit nodes get a working copy (set by the host together with the instantiation)
-  int inline_fix;          // the last CTA of the check kernel also recomputes the sums of located / fallen-back
-                           // nodes (small batches, at most one parity, sums wanted): no fix kernel follows
-  int out_act;             // forward sums: activation applied as they are written (step C1), or identity
-  const float* out_mask;   // backward sums: zeroed where this input is not positive (step C2), or NULL
-  uint32_t* bump;          // iteration counter of the fault plans to advance when the kernel ends, or NULL
-};
-
-struct PhaseGeom {
-  int n_cw, K, kd, r, len, nsl, slen;
-  size_t n_el;
-  const float* P;
-};
-
-__device__ __forceinline__ PhaseGeom phase_geom(const Geom& g, int phase, int B) {
-  PhaseGeom q;
-  if (phase == CODENET_PHASE_FWD) {
-    q.n_cw = g.n; q.K = g.M; q.kd = g.m; q.r = g.r_row; q.len = g.b_r; q.nsl = g.ns; q.slen = g.T; q.P = g.Pr;
-  } else {
-    q.n_cw = g.m; q.K = g.Nn; q.kd = g.n; q.r = g.r_col; q.len = g.b_c; q.nsl = g.nsc; q.slen = g.Tc; q.P = g.Pc;
-  }
-  q.n_el = (size_t)q.len * B;
-  return q;
-}
-
-// A sum on its way out: s -> f(s) for the feedforward sums, c -> c * [x > 0] for the backpropagated ones.
-__device__ __forceinline__ float finish_out(const CheckParams& p, float acc, size_t idx) {
-  if (p.out_act == CODENET_ACT_RELU && acc < 0.0f) acc = 0.0f;
-  if (p.out_mask != nullptr && !(p.out_mask[idx] > 0.0f)) acc = 0.0f;
-  return acc;
-}
-
-// The noise of one element of a hit node, as a real call: hit nodes are rare, and every inlined copy of the
-// generator is a few kilobytes of instructions that the clean path would have to fetch past.
-__device__ __noinline__ float hit_noise(uint32_t seed, uint32_t key1, uint32_t iteration, uint32_t node_id, uint32_t e,
-                                        float sigma) {
-  return soft_error_noise(seed, key1, iteration, node_id, e, sigma);
-}
-
-__device__ __forceinline__ float clean_value(const CheckParams& p, const PhaseGeom& q, int cw, int k, size_t e) {
-  if (p.src_kind == 0) return p.src[((size_t)cw * q.K + k) * q.n_el + e];
-  if (p.src_kind == 2) {  // feedforward partials of the column strips of block-column cw, fixed order
-    float v = 0.0f;
-    for (int s = 0; s < p.spb; ++s) v += p.src[((size_t)(cw * p.spb + s) * p.g.Mbr) * p.B + (size_t)k * q.n_el + e];
-    return v;
-  }
-  const int pos = (int)(e / p.B), b = (int)(e % p.B);
-  const float* s0 = p.src + ((size_t)cw * p.RT * p.B + b) * p.g.ld + (size_t)k * p.g.ldb + pos;
-  const size_t step = (size_t)p.B * p.g.ld;
-  // fixed summation order (row tiles in increasing order), loads issued sixteen at a time
-  float v = 0.0f;
-  int rt = 0;
-  for (; rt + 16 <= p.RT; rt += 16) {
-    float a[16];
-#pragma unroll
-    for (int w = 0; w < 16; ++w) a[w] = s0[(size_t)(rt + w) * step];
-#pragma unroll
-    for (int w = 0; w < 16; ++w) v += a[w];
-  }
-  for (; rt + 4 <= p.RT; rt += 4) {
-    const float a0 = s0[(size_t)rt * step], a1 = s0[(size_t)(rt + 1) * step];
-    const float a2 = s0[(size_t)(rt + 2) * step], a3 = s0[(size_t)(rt + 3) * step];
-    v = (((v + a0) + a1) + a2) + a3;
-  }
-  for (; rt < p.RT; ++rt) v += s0[(size_t)rt * step];
-  return v;
-}
-
-// clean_value for four elements of one node at a time: the same sums in the same order, with the partials of
-// all four (eight rows of partials per round) in flight together.  Elements that are not wanted repeat e[0].
-__device__ __forceinline__ void clean_value4(const CheckParams& p, const PhaseGeom& q, int cw, int k,
-                                             const size_t (&e)[4], float (&v)[4]) {
-  if (p.src_kind == 0) {
-#pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = p.src[((size_t)cw * q.K + k) * q.n_el + e[u]];
-    return;
-  }
-  const float* s0[4];
-  size_t step;
-  int np;
-  if (p.src_kind == 2) {
-#pragma unroll
-    for (int u = 0; u < 4; ++u) s0[u] = p.src + ((size_t)cw * p.spb * p.g.Mbr) * p.B + (size_t)k * q.n_el + e[u];
-    step = (size_t)p.g.Mbr * p.B;
-    np = p.spb;
-  } else {
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int pos = (int)(e[u] / p.B), b = (int)(e[u] % p.B);
-      s0[u] = p.src + ((size_t)cw * p.RT * p.B + b) * p.g.ld + (size_t)k * p.g.ldb + pos;
-    }
-    step = (size_t)p.B * p.g.ld;
-    np = p.RT;
-  }
-#pragma unroll
-  for (int u = 0; u < 4; ++u) v[u] = 0.0f;
-  int r = 0;
-  for (; r + 8 <= np; r += 8) {
-    float a[4][8];
-#pragma unroll
-    for (int w = 0; w < 8; ++w)
-#pragma unroll
-      for (int u = 0; u < 4; ++u) a[u][w] = s0[u][(size_t)(r + w) * step];
-#pragma unroll
-    for (int w = 0; w < 8; ++w)
-#pragma unroll
-      for (int u = 0; u < 4; ++u) v[u] += a[u][w];
-  }
-  for (; r < np; ++r)
-#pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] += s0[u][(size_t)r * step];
-}
-
-__device__ __forceinline__ uint32_t node_id_of(const Geom& g, int phase, int cw, int k) {
-  const int i = phase == CODENET_PHASE_FWD ? k : cw, j = phase == CODENET_PHASE_FWD ? cw : k;
-  return (uint32_t)(i * g.Nn + j);
-}
-
-// Which nodes of every codeword the injection plan hits, into shared memory.
-__device__ void build_hit_masks(const CheckParams& p, const PhaseGeom& q, unsigned long long* s_inj) {
-  for (int t = threadIdx.x; t < MAXN; t += blockDim.x) s_inj[t] = 0ull;
-  __syncthreads();
-  if (p.fault.mode != CODENET_FAULT_NONE) {
-    const uint32_t it = p.fault.iteration ? *p.fault.iteration : 0u;
-    const bool fwd = p.phase == CODENET_PHASE_FWD;
-    const uint32_t n_active = (uint32_t)(q.n_cw * q.K);
-    for (int t = threadIdx.x; t < q.n_cw * q.K; t += blockDim.x) {
-      const int cw = t / q.K, k = t % q.K;
-      const int i = fwd ? k : cw, j = fwd ? cw : k;
-      const uint32_t node_id = (uint32_t)(i * p.g.Nn + j);
-      const uint32_t active = fwd ? (uint32_t)(i * p.g.n + j) : node_id;
-      if (node_is_hit(p.fault, (uint32_t)p.phase, it, node_id, active, n_active))
-        atomicOr(&s_inj[cw], 1ull << k);
-    }
-  }
-  __syncthreads();
-}
-
-__device__ __forceinline__ float block_max256(float v, float* red) {
-  v = warp_max(v);
-  __syncthreads();
-  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
-  __syncthreads();
-  float m = 0.0f;
-#pragma unroll
-  for (int w = 0; w < CK_WARPS; ++w) m = fmaxf(m, red[w]);
-  return m;
-}
-
-// Inverse of an s x s matrix (s <= 4), Gaussian elimination with partial pivoting, in double.
-__device__ bool invert_small(int s, const double* A, double* inv) {
-  double a[MAXR][2 * MAXR];
-  for (int r = 0; r < s; ++r)
-    for (int c = 0; c < s; ++c) {
-      a[r][c] = A[r * s + c];
-      a[r][s + c] = r == c ? 1.0 : 0.0;
-    }
-  for (int pv = 0; pv < s; ++pv) {
-    int best = pv;
-    for (int r = pv + 1; r < s; ++r)
-      if (fabs(a[r][pv]) > fabs(a[best][pv])) best = r;
-    if (a[best][pv] == 0.0) return false;
-    if (best != pv)
-      for (int c = 0; c < 2 * s; ++c) {
-        const double t = a[pv][c]; a[pv][c] = a[best][c]; a[best][c] = t;
-      }
-    const double piv = a[pv][pv];
-    for (int c = 0; c < 2 * s; ++c) a[pv][c] /= piv;
-    for (int r = 0; r < s; ++r) {
-      if (r == pv) continue;
-      const double f = a[r][pv];
-      if (f == 0.0) continue;
-      for (int c = 0; c < 2 * s; ++c) a[r][c] -= f * a[pv][c];
-    }
-  }
-  for (int r = 0; r < s; ++r)
-    for (int c = 0; c < s; ++c) inv[r * s + c] = a[r][s + c];
-  return true;
-}
-
-// The outputs of one codeword as the checks see them.  Small batches copy every node output into the
-// working copy; large batches copy only the nodes the injection plan hits (the others are read where
-// the product kernel left them), so `own` says which nodes live in the working copy.
-struct CwView {
-  const float* yw;          // working copy of the codeword
-  const float* ys;          // clean source of the codeword (same layout)
-  unsigned long long own;   // bit k: node k is read from the working copy
-  __device__ __forceinline__ float at(const PhaseGeom& q, int k, size_t e) const {
-    return (((own >> k) & 1ull) ? yw : ys)[(size_t)k * q.n_el + e];
-  }
-};
-
-__device__ __forceinline__ bool lazy_copy(const CheckParams& p) {
-  return p.lazy != 0;   // decided on the host: large batch, node outputs read in place, 16-byte aligned buffers
-}
-
-__device__ __forceinline__ CwView cw_view(const CheckParams& p, const PhaseGeom& q, const unsigned long long* s_inj,
-                                          int cw) {
-  CwView v;
-  v.yw = p.Yw + (size_t)cw * q.K * q.n_el;
-  if (lazy_copy(p)) { v.ys = p.src + (size_t)cw * q.K * q.n_el; v.own = s_inj[cw]; }
-  else { v.ys = v.yw; v.own = ~0ull; }
-  return v;
-}
-
-// Syndrome of one element: syn[q] = sum_k P[k,q] out_k - out_{kd+q}.
-__device__ __forceinline__ void syndrome_at(const CwView& yw, const PhaseGeom& q, const float* sP, size_t e,
-                                            float (&syn)[MAXR]) {
-#pragma unroll
-  for (int t = 0; t < MAXR; ++t) syn[t] = t < q.r ? -yw.at(q, q.kd + t, e) : 0.0f;
-  for (int k = 0; k < q.kd; ++k) {
-    const float o = yw.at(q, k, e);
-#pragma unroll
-    for (int t = 0; t < MAXR; ++t)
-      if (t < q.r) syn[t] = fmaf(sP[k * q.r + t], o, syn[t]);
-  }
-}
-
-// Erasure decoding of one element under a plan: the located data outputs are solved from the
-// lowest-indexed unlocated parities; par[] receives every parity re-encoded from the result.
-__device__ __forceinline__ void decode_at(const CwView& yw, const PhaseGeom& q, const float* sP, const CwPlan& pl,
-                                          size_t e, float (&fix)[MAXR], double (&par)[MAXR]) {
-  double rhs[MAXR];
-#pragma unroll
-  for (int a = 0; a < MAXR; ++a) rhs[a] = a < pl.nfd ? (double)yw.at(q, q.kd + pl.q[a], e) : 0.0;
-#pragma unroll
-  for (int t = 0; t < MAXR; ++t) par[t] = 0.0;
-  for (int k = 0; k < q.kd; ++k) {
-    if ((pl.F >> k) & 1ull) continue;
-    const double o = (double)yw.at(q, k, e);
-#pragma unroll
-    for (int a = 0; a < MAXR; ++a)
-      if (a < pl.nfd) rhs[a] -= (double)sP[k * q.r + pl.q[a]] * o;
-#pragma unroll
-    for (int t = 0; t < MAXR; ++t)
-      if (t < q.r) par[t] += (double)sP[k * q.r + t] * o;
-  }
-#pragma unroll
-  for (int a = 0; a < MAXR; ++a) {
-    double acc = 0.0;
-#pragma unroll
-    for (int b = 0; b < MAXR; ++b)
-      if (a < pl.nfd && b < pl.nfd) acc += pl.ainv[a * pl.nfd + b] * rhs[b];
-    fix[a] = (float)acc;
-  }
-#pragma unroll
-  for (int a = 0; a < MAXR; ++a)
-    if (a < pl.nfd) {
-#pragma unroll
-      for (int t = 0; t < MAXR; ++t)
-        if (t < q.r) par[t] += (double)sP[pl.fd[a] * q.r + t] * (double)fix[a];
-    }
-}
-
-// Report from the per-codeword plans; called by every thread of one CTA (>= 64 threads).
-// s_a / s_b: two shared float arrays of MAXN entries used as scratch.
-__device__ void write_report(const CheckParams& p, int n_cw, const unsigned* final_state, float* s_a, float* s_b) {
-  __shared__ unsigned s_cnt[4];
-  __shared__ unsigned long long s_dmask;
-  codenet_report_t* rep = p.rep;
-  const int cw = threadIdx.x;
-  if (cw < 4) s_cnt[cw] = 0u;
-  if (cw == 0) s_dmask = 0ull;
-  __syncthreads();
-  if (cw < MAXN) {
-    float mn = FLT_MAX, mx = 0.0f;
-    if (cw < n_cw) {
-      const volatile CwPlan& pl = p.plan[cw];  // written by other CTAs of this grid
-      const int state = final_state ? (int)final_state[cw] : pl.state;
-      uint32_t outcome = CODENET_CLEAN;
-      if (state == 1) outcome = CODENET_CORRECTED;
-      else if (state == 3) outcome = p.have_clean ? CODENET_FALLBACK : CODENET_FAILED;
-      const unsigned long long F = pl.F;
-      rep->flagged_mask[cw] = pl.detected ? F : 0ull;
-      rep->injected_mask[cw] = pl.injected;
-      if (pl.detected) {
-        atomicOr(&s_dmask, 1ull << cw);
-        atomicAdd(&s_cnt[0], 1u);
-        atomicAdd(&s_cnt[1], (unsigned)__popcll(F));
-      }
-      if (state == 3) atomicAdd(&s_cnt[2], 1u);
-      atomicMax(&s_cnt[3], outcome);
-      mn = pl.min_hit;
-      mx = pl.max_clean;
-    } else {
-      rep->flagged_mask[cw] = 0;
-      rep->injected_mask[cw] = 0;
-    }
-    s_a[cw] = mn;
-    s_b[cw] = mx;
-  }
-  __syncthreads();
-  if (cw == 0) {
-    float mn = FLT_MAX, mx = 0.0f;
-    for (int k = 0; k < MAXN; ++k) { mn = fminf(mn, s_a[k]); mx = fmaxf(mx, s_b[k]); }
-    rep->status = (p.tc_flag && *p.tc_flag) ? (uint32_t)CODENET_TIMEOUT : s_cnt[3];
-    rep->n_detected_cw = s_cnt[0];
-    rep->n_flagged_nodes = s_cnt[1];
-    rep->n_fallback_cw = s_cnt[2];
-    rep->detected_mask = s_dmask;
-    rep->min_margin_hit = mn;
-    rep->max_margin_clean = mx;
-  }
-  __syncthreads();
-}
-
-// Sum over codewords of the data-node outputs: s_i = sum_j y_ij (forward), c_j = sum_i z_ij (backward).
-__device__ __forceinline__ void output_index(const Geom& g, bool fwd, int gidx, int* node, int* pos) {
-  const int len = fwd ? g.b_r : g.b_c;
-  *node = gidx / len;
-  *pos = gidx % len;
-}
-
-#ifdef CODENET_PHASE_TIMING
-__device__ unsigned long long g_phase_ts[16];
-__device__ unsigned long long g_phase_cta[16][1024];   // every CTA's stamps, for the spread across the grid
-#define PHASE_TS(k) do { if (threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); if (blockIdx.x == 0) g_phase_ts[k] = t_; if (blockIdx.x < 1024) g_phase_cta[k][blockIdx.x] = t_; } } while (0)
-#else
-#define PHASE_TS(k) do { } while (0)
-#endif
 
 // Sums over the 32 lanes of 32 values per lane (v[a][b], index a * 8 + b) with 31 shuffles: at every
 // step a lane keeps the half of its values whose index bit matches its lane bit and hands the other
@@ -678,34 +335,14 @@ __device__ __forceinline__ void big_phase_x_wide(const CheckParams& p, const Pha
   }
 }
 
-// Value of data node `node` of codeword `cw` at element e after decoding / fallback.
-__device__ __forceinline__ float final_value(const CheckParams& p, const PhaseGeom& q, const float* sP,
-                                             const unsigned long long* s_inj, const unsigned* s_final, int cw,
-                                             int node, size_t e) {
-  const CwView yw = cw_view(p, q, s_inj, cw);
-  const int state = (int)s_final[cw];
-  if (state == 0) return yw.at(q, node, e);
-  if (state == 1) {
-    const CwPlan& pl = p.plan[cw];
-    if (!((pl.F >> node) & 1ull)) return yw.at(q, node, e);
-    float fix[MAXR];
-    double par[MAXR];
-    decode_at(yw, q, sP, pl, e, fix, par);
-    float v = 0.0f;
-#pragma unroll
-    for (int a = 0; a < MAXR; ++a)
-      if (a < pl.nfd && pl.fd[a] == node) v = fix[a];
-    return v;
-  }
-  // uncorrectable: the fault-free recomputation, when there is one
-  if (p.have_clean && ((s_inj[cw] >> node) & 1ull)) return clean_value(p, q, cw, node, e);
-  return yw.at(q, node, e);
-}
-
 template <bool BIG>
 __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
   cg::grid_group grid = cg::this_grid();
-  PHASE_TS(0);
+  // which statistics buffer this call works in: read by every CTA before the first grid barrier, flipped by
+  // CTA 0 after the second
+  const int st_par = __ldcg(p.parity) & 1;
+  p.st = p.st_base + st_par;
+  p.st_next = p.st_base + (st_par ^ 1);
   const Geom& g = p.g;
   const bool fwd = p.phase == CODENET_PHASE_FWD;
   const PhaseGeom q = phase_geom(g, p.phase, p.B);
@@ -741,7 +378,6 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
   }
   const uint32_t it = p.fault.iteration ? *p.fault.iteration : 0u;
   const uint32_t key1 = (p.fault.layer << 8) | (uint32_t)p.phase;
-  PHASE_TS(1);
 
   // ------------------------------------------------------------------------------------------
   // phase U: one warp per (codeword, node, slice): working copy, node norm, inner-checksum ratio
@@ -890,7 +526,6 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       }
       if (lane == 0) atomicMax(&p.st->ratio[cw * MAXN + k], __float_as_uint(worst));
     }
-    PHASE_TS(7);
     if (big_batch && node_check) {
       // checksum side of the inner check, u.x or v.delta: a warp takes four units of one codeword (they
       // share the vector operand) and eight batch entries, lanes along the dot-product index
@@ -949,9 +584,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       }
     }
   }
-  PHASE_TS(2);
   grid.sync();
-  PHASE_TS(3);
 
   // ------------------------------------------------------------------------------------------
   // phase X: syndrome maxima; sums assuming no error; inner-checksum update; reset of the
@@ -1028,7 +661,6 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     for (int cw = tid; cw < q.n_cw; cw += CK_THREADS)
       if (s_syn[cw]) atomicMax(&p.st->syn[cw], s_syn[cw]);
   }
-  PHASE_TS(8);
   if (big_batch && one_pass) {
     __shared__ float s_sums[BIG_KD][BIG_TR][33];
     if (q.kd <= 8) {
@@ -1164,7 +796,6 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       }
     }
   }
-  PHASE_TS(9);
   if (p.update_checksums && big_batch && B >= 128) {
     // batches of 128 and more: u_ij += lr sum_b (1^T delta~_i)[b] x~_j[b][:] and
     // v_ij += lr sum_b (x~_j^T 1)[b] delta~_i[b][:], with the row loads shared between blocks (a batch this long
@@ -1312,9 +943,8 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     }
     for (int c = q.n_cw + tid; c < MAXN; c += CK_THREADS) { r->flagged_mask[c] = 0ull; r->injected_mask[c] = 0ull; }
   }
-  PHASE_TS(4);
   grid.sync();
-  PHASE_TS(5);
+  if (blockIdx.x == 0 && tid == 0) *p.parity = st_par ^ 1;
 
   // ------------------------------------------------------------------------------------------
   // phase D: one CTA per codeword decides
@@ -1330,7 +960,6 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     }
     if (tid == MAXN) s_smax = __uint_as_float(__ldcg(&p.st->syn[cw]));
     __syncthreads();
-    PHASE_TS(10);
     // scale: the (r+1)-th largest node norm, so that up to r corrupted outputs cannot inflate it.  Every
     // node's thread counts the norms that come before its own in decreasing order (ties by index); the
     // one with exactly r before it holds the scale.
@@ -1372,7 +1001,6 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       else s_state = 3;
       }
     __syncthreads();
-    PHASE_TS(11);
     int state = s_state;  // block-uniform copy
     const bool detected = state != 0;
 
@@ -1456,7 +1084,6 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       state = found ? 1 : 3;
     }
 
-    PHASE_TS(12);
     if (tid == 0) {
       CwPlan& pl = p.plan[cw];
       const unsigned long long F = s_F;
@@ -1567,25 +1194,13 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
   }
   // every CTA read the counter before the first grid barrier
   if (p.bump != nullptr && blockIdx.x == 0 && tid == 0) *p.bump += 1u;
-  PHASE_TS(6);
 }
-#ifdef CODENET_PHASE_TIMING
-}  // namespace
-extern "C" void codenet_debug_phase_ts(unsigned long long* out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, g_phase_ts, sizeof(unsigned long long) * 16);
-}
-extern "C" void codenet_debug_phase_cta(unsigned long long* out) {   // [16][1024]
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(out, g_phase_cta, sizeof(unsigned long long) * 16 * 1024);
-}
-namespace {
-#endif
 
 // SPARE: some plan may have a spare parity to be verified on (two and more parities in the phase's code);
 // that pass needs a grid barrier, so only this instantiation is a cooperative launch.
 template <bool SPARE>
 __global__ void __launch_bounds__(CK_THREADS) fix_kernel(CheckParams p) {
+  p.st = p.st_base + ((__ldcg(p.parity) & 1) ^ 1);   // the buffer the check kernel before this one worked in
   if (p.st->need_fix == 0u) return;  // the usual case: every codeword passed its checks
   const Geom& g = p.g;
   const bool fwd = p.phase == CODENET_PHASE_FWD;
@@ -1698,12 +1313,14 @@ __global__ void __launch_bounds__(CK_THREADS) fix_kernel(CheckParams p) {
   }
 }
 
-// Plain sums of the data-node outputs for layers that run no check at all.
-__global__ void __launch_bounds__(CK_THREADS)
-sum_outputs_kernel(Geom g, int phase, int B, const float* __restrict__ Y, float* __restrict__ out, int out_act,
-                   codenet_report_t* rep) {
-  const bool fwd = phase == CODENET_PHASE_FWD;
-  const PhaseGeom q = phase_geom(g, phase, B);
+// Plain sums of the data-node outputs for calls that check nothing (no code, or the checks switched off, and no
+// injection): s_i = sum_j y_ij / c_j = sum_i z_ij straight from the node outputs or their partial sums, in the same
+// fixed order as the checked path, an empty report.  No barrier, no working copy, no inner-checksum update.
+__global__ void __launch_bounds__(CK_THREADS) sum_outputs_kernel(CheckParams p) {
+  const Geom& g = p.g;
+  const bool fwd = p.phase == CODENET_PHASE_FWD;
+  const PhaseGeom q = phase_geom(g, p.phase, p.B);
+  const int B = p.B;
   const int nout = fwd ? g.n_out : g.n_in;
   for (size_t idx = blockIdx.x * (size_t)CK_THREADS + threadIdx.x; idx < (size_t)nout * B;
        idx += (size_t)gridDim.x * CK_THREADS) {
@@ -1711,15 +1328,20 @@ sum_outputs_kernel(Geom g, int phase, int B, const float* __restrict__ Y, float*
     int node, pos;
     output_index(g, fwd, gidx, &node, &pos);
     float acc = 0.0f;
-    for (int cw = 0; cw < q.n_cw; ++cw) acc += Y[(((size_t)cw * q.K + node) * q.len + pos) * B + b];
-    if (out_act == CODENET_ACT_RELU && acc < 0.0f) acc = 0.0f;
-    out[(size_t)b * nout + gidx] = acc;
+    for (int cw = 0; cw < q.n_cw; ++cw) acc += clean_value(p, q, cw, node, (size_t)pos * B + b);
+    const size_t oi = (size_t)b * nout + gidx;
+    p.out[oi] = finish_out(p, acc, oi);
   }
-  if (rep && blockIdx.x == 0 && threadIdx.x == 0) {
-    rep->status = CODENET_CLEAN; rep->n_detected_cw = 0; rep->n_flagged_nodes = 0; rep->n_fallback_cw = 0;
-    rep->detected_mask = 0; rep->min_margin_hit = FLT_MAX; rep->max_margin_clean = 0.0f;
-    for (int cw = 0; cw < MAXN; ++cw) { rep->flagged_mask[cw] = 0; rep->injected_mask[cw] = 0; }
+  codenet_report_t* rep = p.rep;
+  if (rep && blockIdx.x == 0) {
+    if (threadIdx.x == 0) {
+      rep->status = (p.tc_flag && *p.tc_flag) ? (uint32_t)CODENET_TIMEOUT : (uint32_t)CODENET_CLEAN;
+      rep->n_detected_cw = 0; rep->n_flagged_nodes = 0; rep->n_fallback_cw = 0;
+      rep->detected_mask = 0; rep->min_margin_hit = FLT_MAX; rep->max_margin_clean = 0.0f;
+    }
+    for (int cw = threadIdx.x; cw < MAXN; cw += CK_THREADS) { rep->flagged_mask[cw] = 0; rep->injected_mask[cw] = 0; }
   }
+  if (p.bump != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *p.bump += 1u;
 }
 
 int g_coop_blocks_check = 0, g_coop_blocks_fix = 0, g_coop_blocks_check_max = 0;
@@ -1772,9 +1394,7 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
   else { p.fault.seed = 0; p.fault.layer = 0; p.fault.mode = CODENET_FAULT_NONE; p.fault.p_q32 = 0; p.fault.sigma = 0.0f; p.fault.iteration = nullptr; }
   p.src = src; p.Yw = Yw; p.Vraw = Vraw; p.out = out;
   p.Xt = L.ws.Xt; p.Dt = L.ws.Dt; p.dsum = L.ws.dsum; p.xsum = L.ws.xsum;
-  const int par = L.check_parity & 1;
-  L.check_parity ^= 1;
-  p.st = L.ws.stats + par; p.st_next = L.ws.stats + (par ^ 1);
+  p.st = nullptr; p.st_next = nullptr; p.st_base = L.ws.stats; p.parity = L.ws.tc_flag + 1;
   p.plan = L.ws.plan; p.rep = rep; p.tc_flag = L.ws.tc_flag; p.chk = L.ws.chk;
   p.out_act = phase == CODENET_PHASE_FWD ? L.out_act : CODENET_ACT_IDENTITY;
   p.out_mask = phase == CODENET_PHASE_BWD ? L.out_mask : nullptr;
@@ -1782,6 +1402,21 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
 
   const Geom& g = L.g;
   const bool fwd = phase == CODENET_PHASE_FWD;
+  const bool phase_unchecked = g.locate_mode == CODENET_LOCATE_OFF ||
+                               ((fwd ? g.r_row : g.r_col) == 0 && g.locate_mode != CODENET_LOCATE_NODECHECK);
+  if (fault == nullptr && out != nullptr && have_clean && !commit && phase_unchecked &&
+      (!update_checksums || !keeps_checksums(g))) {
+    // nothing to inject and nothing to decide: the sums alone, one plain launch (the inner checksums are left
+    // alone where nothing can read them: keeps_checksums)
+    p.bump = nullptr;
+    if (L.bump_after != nullptr && !fwd) { p.bump = L.bump_after; L.bump_done = true; }
+    const size_t n = (size_t)(fwd ? g.n_out : g.n_in) * B;
+    size_t blocks = (n + CK_THREADS - 1) / CK_THREADS;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    sum_outputs_kernel<<<(int)(blocks < 1 ? 1 : blocks), CK_THREADS, 0, st>>>(p);
+    count_launch();
+    return cudaGetLastError();
+  }
   const int n_cw = fwd ? g.n : g.m, K = fwd ? g.M : g.Nn, nsl = fwd ? g.ns : g.nsc;
   const size_t n_el = (size_t)(fwd ? g.b_r : g.b_c) * B;
   // enough CTAs for one warp per unit and one thread per element, within the co-resident limit
@@ -1834,11 +1469,14 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
 
 cudaError_t launch_sum_outputs(const Geom& g, int phase, int B, const float* Y, float* out, int out_act,
                                codenet_report_t* rep, cudaStream_t st) {
+  CheckParams p;
+  memset(&p, 0, sizeof(p));
+  p.g = g; p.phase = phase; p.B = B; p.src = Y; p.src_kind = 0; p.out = out; p.rep = rep; p.out_act = out_act;
   const size_t n = (size_t)(phase == CODENET_PHASE_FWD ? g.n_out : g.n_in) * B;
   size_t blocks = (n + CK_THREADS - 1) / CK_THREADS;
   if (blocks > 148 * 8) blocks = 148 * 8;
   if (blocks < 1) blocks = 1;
-  sum_outputs_kernel<<<(int)blocks, CK_THREADS, 0, st>>>(g, phase, B, Y, out, out_act, rep);
+  sum_outputs_kernel<<<(int)blocks, CK_THREADS, 0, st>>>(p);
   count_launch();
   return cudaGetLastError();
 }
