@@ -37,7 +37,10 @@ def _peaks():
 
 
 class ClockSampler(threading.Thread):
-    """Samples SM clocks and throttle reasons through NVML (read-only) while the timed region runs."""
+    """Samples SM clocks and throttle reasons while the timed region runs: through NVML when the Python
+    binding is there, otherwise from a read-only ``nvidia-smi --query-gpu`` loop.  Nothing is ever set."""
+
+    NAMES = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index, period=0.01):
         super().__init__(daemon=True)
@@ -46,29 +49,62 @@ class ClockSampler(threading.Thread):
         self.sm = []
         self.reason_bits = 0
         self.sm_max = None
+        self.source = None
         self.stop_flag = threading.Event()
+
+    def _run_nvml(self):
+        import pynvml as nv
+        nv.nvmlInit()
+        h = nv.nvmlDeviceGetHandleByIndex(self.index)
+        self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+        self.source = "nvml"
+        while not self.stop_flag.is_set():
+            self.sm.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+            self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+            self.stop_flag.wait(self.period)
+
+    def _run_smi(self):
+        uuid = None
+        try:
+            import torch
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(self.index).uuid)
+        except Exception:
+            pass
+        cmd = ["nvidia-smi", "--query-gpu=clocks.sm,clocks.max.sm,clocks_event_reasons.active",
+               "--format=csv,noheader,nounits", "-lms", "100", "-i", uuid or str(self.index)]
+        proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        self.source = "nvidia-smi"
+        try:
+            while not self.stop_flag.is_set():
+                row = proc.stdout.readline()
+                if not row:
+                    break
+                f = [x.strip() for x in row.split(",")]
+                try:
+                    self.sm.append(float(f[0]))
+                    self.sm_max = float(f[1])
+                    self.reason_bits |= int(f[2], 16)
+                except (ValueError, IndexError):
+                    continue
+        finally:
+            proc.terminate()
 
     def run(self):
         try:
-            import pynvml as nv
-            nv.nvmlInit()
-            h = nv.nvmlDeviceGetHandleByIndex(self.index)
-            self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
-            while not self.stop_flag.is_set():
-                self.sm.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
-                self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
-                self.stop_flag.wait(self.period)
-        except Exception as exc:  # NVML missing: fall back to one nvidia-smi sample
-            self.error = str(exc)
+            self._run_nvml()
+        except Exception:
+            try:
+                self._run_smi()
+            except Exception as exc:
+                self.error = str(exc)
 
     def summary(self):
         if not self.sm:
             return {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": ["no samples"]}
-        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
-        reasons = [n for bit, n in names.items() if self.reason_bits & bit]
+        reasons = [n for bit, n in self.NAMES.items() if self.reason_bits & bit]
         sm = sorted(self.sm)
         return {"sm_mhz": sm[len(sm) // 2], "sm_min_mhz": sm[0], "sm_max_mhz": self.sm_max, "reasons": reasons,
-                "samples": len(sm)}
+                "samples": len(sm), "source": self.source}
 
 
 def max_over_ranks(seconds, world, device="cuda"):
@@ -86,9 +122,18 @@ def whole_job_value(world, steps, layers, seconds_max):
     return world * steps * layers / seconds_max
 
 
-# DRAM bytes per launch of the dominant kernel on configuration 3, from the ncu capture summarised in
-# profiles/backward_update_kernel_c3.md (dram__bytes_read.sum + dram__bytes_write.sum)
-NCU_TRAFFIC_BYTES = {"c3": 618.3e6}
+def _ncu_traffic(workload):
+    """DRAM bytes per launch of the workload's dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
+    ncu capture), from the table kept in profiles/dram_traffic.md; None where no capture exists."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.md")
+    try:
+        for row in open(path):
+            f = [x.strip() for x in row.strip().strip("|").split("|")]
+            if len(f) >= 3 and f[0] == workload:
+                return float(f[2])
+    except (OSError, ValueError):
+        pass
+    return None
 
 
 def _workload_bytes(sp, esz):
@@ -154,10 +199,16 @@ def _config_dict(cfg, args):
                   % (sum(_workload_bytes(s, 2 if cfg.bf16 else 4)[1] for s in cfg.layers) / 2 / len(cfg.layers) / 1e6)}
 
 
+_WEIGHTS = {}   # host copies of the synthetic weights, so that the comparison legs do not draw them again
+
+
 def build_net(cn, wl, torch, cfg, locate_mode=None, coded=True):
     layers = []
     for l, sp in enumerate(cfg.layers):
-        W = wl.weights(sp.n_out, sp.n_in, seed=cfg.seed, layer=l, bf16=cfg.bf16)
+        key = (cfg.name, l, sp.n_out, sp.n_in, cfg.seed, cfg.bf16)
+        if key not in _WEIGHTS:
+            _WEIGHTS[key] = wl.weights(sp.n_out, sp.n_in, seed=cfg.seed, layer=l, bf16=cfg.bf16)
+        W = _WEIGHTS[key]
         Wd = torch.tensor(W, device="cuda").to(torch.bfloat16 if cfg.bf16 else torch.float32)
         rr, rc = (sp.r_row, sp.r_col) if coded else (0, 0)
         Pr, Pc = (wl.layer_codes(sp, cfg.seed, l) if (sp.gaussian_code and coded) else (None, None))
@@ -291,6 +342,113 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
     return secs, launched, bytes_in, bytes_out
 
 
+def _stats(vals):
+    v = sorted(vals)
+    return {"ms": v[len(v) // 2], "ms_min": v[0], "ms_max": v[-1], "repeats": len(v)}
+
+
+def overhead_legs(cn, wl, torch, cfg, la, steps, repeats):
+    """Detect / decode overhead = (T_coded - T_coded,checks-off) / T_uncoded and the cost of the redundant blocks
+    alone, T_checks-off / T_uncoded - 1.  Each leg is timed like the headline value: recorded steps replayed
+    `steps` times, `repeats` times over; the median counts, the spread is printed.  The checks-off and uncoded
+    legs launch no check kernel at all (their sums come from one plain reduction kernel)."""
+    legs = {}
+    for name, kw in (("coded", {}), ("checks_off", {"locate_mode": cn.LOCATE_OFF}),
+                     ("uncoded", {"coded": False, "locate_mode": cn.LOCATE_OFF})):
+        ls, nt = build_net(cn, wl, torch, cfg, **kw)
+        times, launches = [], 0
+        for _ in range(repeats):
+            sec, launches, _, _ = timed_steps(cn, torch, nt, ls, cfg, wl, steps, 3, name == "coded", lookahead=la, graphs=True)
+            times.append(1e3 * sec / steps)
+        legs[name] = _stats(times)
+        legs[name]["launches_per_step"] = launches / steps
+        nt.free()
+        for lay in ls:
+            lay.free()
+    c, o, u = legs["coded"]["ms"], legs["checks_off"]["ms"], legs["uncoded"]["ms"]
+    worst = (legs["coded"]["ms_max"] - legs["checks_off"]["ms_min"]) / legs["uncoded"]["ms_min"]
+    best = (legs["coded"]["ms_min"] - legs["checks_off"]["ms_max"]) / legs["uncoded"]["ms_max"]
+    return {"ms_coded": c, "ms_checks_off": o, "ms_uncoded": u, "legs": legs, "steps_per_leg": steps,
+            "detect_decode_overhead_pct": 100.0 * (c - o) / u,
+            "detect_decode_overhead_pct_range": [100.0 * best, 100.0 * worst],
+            "redundancy_cost_pct": 100.0 * (o / u - 1.0),
+            "method": "recorded steps, median of %d runs of %d steps per leg" % (repeats, steps)}
+
+
+def p_sweep(cn, wl, torch, cfg, la, steps, count_steps):
+    """Throughput and decision counts at each soft-error probability the configuration names."""
+    import dataclasses
+    rows = []
+    for p in cfg.p_sweep:
+        cfgp = dataclasses.replace(cfg, p=p)
+        ls, nt = build_net(cn, wl, torch, cfgp)
+        L = len(ls)
+        sec, _, _, _ = timed_steps(cn, torch, nt, ls, cfgp, wl, steps, 3, p > 0, lookahead=la, graphs=True)
+        # decisions: a short run that reads every report
+        mode = {"bernoulli": 1, "exactly_one": 2, "none": 0}[cfgp.fault_mode] if p > 0 else 0
+        its = torch.arange(100000, 100000 + count_steps, dtype=torch.int32, device="cuda")
+        reps = cn.new_reports(2 * L)
+        loss_dev = torch.zeros(1, device="cuda")
+        xs = [wl.layer_inputs(cfgp, k) for k in range(4)]
+        dx = [(torch.tensor(a, device="cuda"), torch.tensor(b, device="cuda")) for a, b in xs]
+        det = corr = fb = hit_phases = 0
+        for it in range(count_steps):
+            faults = [cn.make_fault(seed=cfgp.seed, layer=l, mode=mode, p=p, sigma=cfgp.sigma, iteration_dev=its[it:]) for l in range(L)]
+            cn.step(nt, dx[it % 4][0], dx[it % 4][1], cfgp.lr, faults=faults, reps_dev=reps, loss_dev=loss_dev)
+            for r in cn.read_reports(reps):
+                det += r.n_detected_cw
+                fb += r.n_fallback_cw
+                corr += r.n_detected_cw - r.n_fallback_cw
+                hit_phases += 1 if any(r.injected_mask) else 0
+        codewords = count_steps * sum(sp.m + sp.n for sp in cfgp.layers)
+        rows.append({"p": p, "ms_per_step": 1e3 * sec / steps, "layer_iterations_per_s": steps * L / sec,
+                     "phases_with_a_hit_pct": 100.0 * hit_phases / (count_steps * 2 * L),
+                     "detected_codewords": det, "corrected_codewords": corr, "fallback_codewords": fb,
+                     "fallback_rate_per_codeword": fb / codewords, "counted_steps": count_steps})
+        nt.free()
+        for lay in ls:
+            lay.free()
+    return rows
+
+
+def workload_bytes_per_step(cfg, la):
+    """Algorithmic bytes of one step: the forward pass reads the (m + r_row) x n active blocks of each layer, the
+    backward + update pass reads and writes every stored block once; with layer 1's next products taken in the
+    update sweep its forward read drops out."""
+    esz = 2 if cfg.bf16 else 4
+    b = sum(sum(_workload_bytes(sp, esz)) for sp in cfg.layers)
+    if la:
+        b -= _workload_bytes(cfg.layers[0], esz)[0]
+    return b
+
+
+def workload_flops_per_step(cfg):
+    return sum(2.0 * cfg.batch * (-(-s.n_out // s.m)) * (-(-s.n_in // s.n)) *
+               ((s.m + s.r_row) * s.n + s.m * (s.n + s.r_col) + s.m * s.n + s.r_row * s.n + s.r_col * s.m)
+               for s in cfg.layers)
+
+
+def short_workload_leg(cn, wl, torch, name, steps, peak):
+    """A bounded run of another configuration beside the headline one: iterations/s, step bytes / time, tensor
+    TFLOP/s, detect / decode overhead."""
+    cfg = wl.config(name)
+    L = len(cfg.layers)
+    la = cfg.batch <= 8
+    ls, nt = build_net(cn, wl, torch, cfg)
+    sec, launches, _, _ = timed_steps(cn, torch, nt, ls, cfg, wl, steps, 5, True, lookahead=la, graphs=True)
+    nt.free()
+    for lay in ls:
+        lay.free()
+    byts = workload_bytes_per_step(cfg, la)
+    out = {"workload": name, "steps": steps, "ms_per_step": 1e3 * sec / steps, "layer_iterations_per_s": steps * L / sec,
+           "launches_per_step": launches / steps, "bytes_per_step": byts,
+           "step_GBs": byts * steps / sec / 1e9, "step_frac_of_hbm_peak": byts * steps / sec / 1e9 / peak}
+    if cfg.batch >= 64:
+        out["tflops"] = workload_flops_per_step(cfg) * steps / sec / 1e12
+    out["overhead"] = overhead_legs(cn, wl, torch, cfg, la, steps, 1)
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -300,6 +458,7 @@ def main():
     ap.add_argument("--workload", default="c3")
     ap.add_argument("--scale", type=int, default=1, help="divide layer widths (for quick checks only)")
     ap.add_argument("--no-extras", action="store_true", help="skip overhead, CPU-baseline and e2e legs")
+    ap.add_argument("--no-others", action="store_true", help="skip the short legs of the batched configurations")
     ap.add_argument("--no-graphs", action="store_true", help="launch every step kernel by kernel instead of replaying recorded steps")
     ap.add_argument("--no-lookahead", action="store_true",
                     help="do not take layer 1's next feedforward products in the update sweep (3-pass)")
@@ -357,7 +516,7 @@ def main():
     bw_ms, bw_n = cn.profile_read(cn.KERNEL_BACKWARD)
     up_ms, up_n = cn.profile_read(cn.KERNEL_UPDATE)
     cn.profile_enable(False)
-    dominant = "backward_update_kernel"
+    dominant = "backward_update_kernel" if cfg.batch <= 8 else "tc_backward_update_kernel"
     if not bu_n and up_n:
         # batches > 8: products and update are separate kernels; the update (read + write of every
         # stored block) is the dominant one
@@ -370,7 +529,7 @@ def main():
         ach = bu_b / (bu_ms / bu_n * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": ach, "peak": peak,
                     "peak_kind": peak_kind + " copy bandwidth", "unit": "GB/s", "frac": ach / peak,
-                    "traffic": NCU_TRAFFIC_BYTES.get(cfg.name) if args.scale == 1 else None, "bytes_per_launch": bu_b, "ms_per_launch": bu_ms / bu_n}
+                    "traffic": _ncu_traffic(cfg.name) if args.scale == 1 else None, "bytes_per_launch": bu_b, "ms_per_launch": bu_ms / bu_n}
         if fw_n:
             fa = fwd_b / (fw_ms / fw_n * 1e-3) / 1e9
             roofline["forward_kernel"] = {"achieved": fa, "frac": fa / peak, "bytes_per_launch": fwd_b,
@@ -381,13 +540,14 @@ def main():
             ba = (bw_b / L) / (bw_ms / bw_n * 1e-3) / 1e9
             roofline["backward_kernel"] = {"achieved": ba, "frac": ba / peak, "bytes_per_launch": bw_b / L,
                                            "ms_per_launch": bw_ms / bw_n}
-        step_bytes = sum(sum(_workload_bytes(s, esz)) for s in cfg.layers) + (bw_b if bw_n else 0)
-        if la and fw_n * 2 < bu_n:
-            # layer 1's feedforward products come out of the update sweep: its blocks are streamed twice
-            # per iteration (read + write), not three times
-            step_bytes -= _workload_bytes(cfg.layers[0], esz)[0]
+        two_pass = la and fw_n * 2 < bu_n
+        # algorithmic bytes of the step (layers that take the products and the update as two kernels move more
+        # than that: their extra backward read is reported beside it, not counted as useful traffic)
+        step_bytes = workload_bytes_per_step(cfg, two_pass)
+        if bw_n:
+            roofline["extra_bytes_of_unfused_layers"] = bw_b
         roofline["passes"] = "2-pass (next feedforward products of layer 1 fused into the update sweep)" \
-            if la and fw_n * 2 < bu_n else "3-pass"
+            if two_pass else "3-pass"
         roofline["step"] = {"bytes_per_step": step_bytes, "achieved": step_bytes * args.steps / secs / 1e9,
                             "frac": step_bytes * args.steps / secs / 1e9 / peak,
                             "frac_of_8TBs": step_bytes * args.steps / secs / 1e9 / 8000.0}
@@ -396,7 +556,8 @@ def main():
         "metric": "coded_sgd_iterations_per_s_per_layer", "value": value, "unit": "layer-iterations/s",
         "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs_max / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 storage, f32 accumulate" if cfg.bf16 else "f32", "data": "synthetic",
+        "dtype": "bf16 storage, f32 accumulate" if cfg.bf16 else ("f32 storage, tf32 multiply, f32 accumulate" if cfg.batch >= 64 else "f32"),
+        "data": "synthetic",
         "config": _config_dict(cfg, args), "gpu_launches": launches, "roofline": roofline,
     }
 
@@ -406,9 +567,7 @@ def main():
                                  "note": "Table 1: 2000 iterations of the same 784-10^4-10^4-10 network in 2322 s on 38 "
                                          "Amazon EC2 m3.medium nodes, checkpoints every 200 iterations included"}
     if cfg.batch >= 64:
-        flops = sum(2.0 * cfg.batch * (-(-s.n_out // s.m)) * (-(-s.n_in // s.n)) *
-                    ((s.m + s.r_row) * s.n + s.m * (s.n + s.r_col) + s.m * s.n + s.r_row * s.n + s.r_col * s.m)
-                    for s in cfg.layers)
+        flops = workload_flops_per_step(cfg)
         line["tensor"] = {"flops_per_step": flops, "achieved_tflops": flops * args.steps / secs / 1e12,
                           "note": "algorithmic flops of the three products; the small bf16 operands are staged as "
                                   "hi + lo pairs, so the tensor pipe executes up to twice the product flops"}
@@ -492,18 +651,24 @@ def main():
         # ---- detect/decode overhead: coded with checks vs coded without checks vs uncoded ----
         for lay in layers:
             lay.free()
-        ksteps = max(20, min(300, args.steps))
-        res = {}
-        for name, kw in (("coded", {}), ("checks_off", {"locate_mode": cn.LOCATE_OFF}), ("uncoded", {"coded": False, "locate_mode": cn.LOCATE_OFF})):
-            ls, nt = build_net(cn, wl, torch, cfg, **kw)
-            s, _, _, _ = timed_steps(cn, torch, nt, ls, cfg, wl, ksteps, 3, name == "coded", lookahead=la)
-            res[name] = 1e3 * s / ksteps
-            nt.free()
-            for lay in ls:
-                lay.free()
-        line["overhead"] = {"ms_coded": res["coded"], "ms_checks_off": res["checks_off"], "ms_uncoded": res["uncoded"],
-                            "detect_decode_overhead_pct": 100.0 * (res["coded"] - res["checks_off"]) / res["uncoded"],
-                            "redundancy_cost_pct": 100.0 * (res["checks_off"] / res["uncoded"] - 1.0)}
+        ksteps = max(200, min(1000, args.steps))
+        line["overhead"] = overhead_legs(cn, wl, torch, cfg, la, ksteps, 3)
+        # ---- the error-rate sweep the configuration names, with the fallback rate at each rate ----
+        if cfg.p_sweep:
+            try:
+                line["p_sweep"] = p_sweep(cn, wl, torch, cfg, la, max(100, min(300, args.steps)), 100 if cfg.batch <= 8 else 30)
+            except Exception as exc:
+                line["p_sweep"] = {"error": str(exc)[:200]}
+        # ---- the batched configurations beside the headline one (bounded legs) ----
+        if cfg.name == "c3" and args.scale == 1 and not args.no_others:
+            others = {}
+            for name in ("c4", "c5"):
+                try:
+                    others[name] = short_workload_leg(cn, wl, torch, name, 100, peak)
+                except Exception as exc:
+                    others[name] = {"error": str(exc)[:200]}
+                _WEIGHTS.clear()
+            line["other_workloads"] = others
         # ---- CPU baseline: the oracle as it stands, bounded sample, this host's cores ----
         from oracle import oracle as orc
         cores = os.cpu_count() or 1

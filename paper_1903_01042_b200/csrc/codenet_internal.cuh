@@ -131,6 +131,8 @@ struct ProfileScope {
 // ---- launchers (kernels_stream.cu) ----------------------------------------------------------
 cudaError_t launch_forward_products(const Geom& g, const float* x, int ldx, int B, float* Y,
                                     cudaStream_t st);
+cudaError_t launch_forward_products_plain(const Geom& g, const float* x, int ldx, int B, float* Y,
+                                          cudaStream_t st);   // never allocates (no profiling events)
 // xnext != NULL: also produce the next iteration's feedforward partials ynext[strip][coded row][b]
 cudaError_t launch_backward_update_fused(const codenet_layer_impl& L, int B, float lr, float* zpart,
                                          const float* xnext, int ldxn, float* ynext, cudaStream_t st);

@@ -451,6 +451,11 @@ cudaError_t backward_fused_launch(const codenet_layer_impl& L, int B, float lr, 
 
 cudaError_t launch_forward_products(const Geom& g, const float* x, int ldx, int B, float* Y, cudaStream_t st) {
   ProfileScope scope(CODENET_KERNEL_FORWARD, st);
+  return launch_forward_products_plain(g, x, ldx, B, Y, st);
+}
+
+// the same launch without the optional event bracket (which creates events, i.e. allocates, when profiling is on)
+cudaError_t launch_forward_products_plain(const Geom& g, const float* x, int ldx, int B, float* Y, cudaStream_t st) {
   return g.dtype == CODENET_BF16 ? forward_dispatch<__nv_bfloat16>(g, x, ldx, B, Y, st)
                                  : forward_dispatch<float>(g, x, ldx, B, Y, st);
 }

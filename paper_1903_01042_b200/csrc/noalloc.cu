@@ -49,7 +49,7 @@ extern "C" int codenet_matvec_noalloc(const float* W_dev, int rows, int cols, in
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   // every scratch element read by the sum is written by the product kernel of this same call,
   // so nothing has to start at zero
-  if (launch_forward_products(g, x_dev, cols, 1, scratch, st) != cudaSuccess) return CODENET_E_CUDA;
+  if (launch_forward_products_plain(g, x_dev, cols, 1, scratch, st) != cudaSuccess) return CODENET_E_CUDA;
   if (launch_sum_outputs(g, CODENET_PHASE_FWD, 1, scratch, s_dev, CODENET_ACT_IDENTITY, nullptr, st) != cudaSuccess) return CODENET_E_CUDA;
   return CODENET_OK;
 }

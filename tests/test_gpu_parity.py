@@ -601,6 +601,53 @@ def test_recorded_steps_replay_like_plain_steps(cn, orc, lookahead):
     torch.cuda.set_stream(torch.cuda.default_stream())
 
 
+def test_eager_checks_between_replays_of_a_recorded_step(cn, orc):
+    """A recorded step, then an odd number of eager checks on the same layer (an evaluation pass with a fault,
+    a stand-alone detect / decode), then the recorded step again: every replay must still decide like the
+    oracle.  (Each check works in one of two statistics buffers and clears the other; which one is the
+    library's own business, whatever the order of eager calls and replays.)"""
+    cfg = wl.config("c1", scale=2)
+    pairs, gnet, onet = _build_net(cn, orc, cfg)
+    pg, po = pairs[0].g, pairs[0].o
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fg = [cn.make_fault(seed=5, layer=0, mode=cn.FAULT_EXACTLY_ONE, sigma=10.0, iteration_dev=it_dev)]
+    fo = [orc.make_fault(seed=5, layer=0, mode=orc.FAULT_EXACTLY_ONE, sigma=10.0)]
+    ev_it = torch.full((1,), 1000, dtype=torch.int32, device="cuda")
+    fe_g = cn.make_fault(seed=6, layer=0, mode=cn.FAULT_EXACTLY_ONE, sigma=10.0, iteration_dev=ev_it)
+    fe_o = orc.make_fault(seed=6, layer=0, mode=orc.FAULT_EXACTLY_ONE, sigma=10.0)
+    reps = cn.new_reports(2)
+    rep_e = cn.new_reports(1)
+    loss_dev = torch.zeros(1, device="cuda")
+    xbuf = torch.zeros((1, 512), device="cuda")
+    tbuf = torch.zeros((1, 512), device="cuda")
+    inputs = [wl.layer_inputs(cfg, it) for it in range(12)]
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(side)
+    xbuf.copy_(_dev(inputs[0][0])); tbuf.copy_(_dev(inputs[0][1]))
+    cn.step(gnet, xbuf, tbuf, cfg.lr, faults=fg, reps_dev=reps, loss_dev=loss_dev)
+    lo, out_o, reps_o = onet.step(inputs[0][0], inputs[0][1], cfg.lr, fo, 0)
+    assert [r.decisions() for r in cn.read_reports(reps)] == [r.decisions() for r in reps_o]
+    graph = cn.net_capture_step(gnet, xbuf, tbuf, cfg.lr, faults=fg, reps_dev=reps, loss_dev=loss_dev)
+    it_dev.fill_(1)
+    for it in range(1, 11):
+        xbuf.copy_(_dev(inputs[it][0])); tbuf.copy_(_dev(inputs[it][1]))
+        cn.net_replay(gnet, graph)
+        lo, out_o, reps_o = onet.step(inputs[it][0], inputs[it][1], cfg.lr, fo, it)
+        assert [r.decisions() for r in cn.read_reports(reps)] == [r.decisions() for r in reps_o], it
+        assert _rel(gnet.output(1).cpu().numpy(), out_o) <= TOL_F32, it
+        # an odd number of eager checks between two replays: one, or three
+        for k in range(1 if it % 2 else 3):
+            xe = wl.gaussian_inputs(1, 512, seed=77, iteration=10 * it + k)
+            ev_it.fill_(1000 + 10 * it + k)
+            s_g = cn.forward(pg, _dev(xe), fault=fe_g, rep_dev=rep_e)
+            s_o, rep_o = po.forward(xe, fe_o, 1000 + 10 * it + k)
+            assert cn.read_reports(rep_e)[0].decisions() == rep_o.decisions(), (it, k)
+            assert _rel(s_g.cpu().numpy(), s_o) <= TOL_F32, (it, k)
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(torch.cuda.default_stream())
+
+
 # ---------------------------------------------------------------------------------------------
 # faults in the stored blocks and regeneration of a block from its code
 # ---------------------------------------------------------------------------------------------

@@ -62,3 +62,32 @@ def test_rejects_what_does_not_fit_the_fixed_scratch(cn):
     with pytest.raises(cn.CodenetError):
         cn.matvec_noalloc(torch.zeros((8, 30), device="cuda"), 3, torch.zeros(30, device="cuda"),
                           torch.zeros(8, device="cuda"))   # block width not a multiple of 4
+
+
+def test_a_warmed_up_call_allocates_nothing_even_while_kernels_are_being_timed(cn):
+    """Free device memory and torch's own allocator count stay where they were across calls, also with the
+    library's per-kernel timing switched on (its event brackets are the one thing in the forward launch that
+    would allocate)."""
+    rows, cols, n_blocks = 512, 1024, 4
+    W = torch.tensor(wl.weights(rows, cols, seed=27), device="cuda")
+    x = torch.tensor(wl.gaussian_inputs(1, cols, seed=28), device="cuda")
+    s = torch.empty(rows, device="cuda")
+    cn.matvec_noalloc(W, n_blocks, x, s)                # first call on the device: looks up the scratch address
+    torch.cuda.synchronize()
+    for timed in (False, True):
+        cn.profile_enable(timed)
+        try:
+            free0, _ = torch.cuda.mem_get_info()
+            held0 = torch.cuda.memory_allocated()
+            before = cn.profile_read(cn.KERNEL_FORWARD)[1] if timed else 0
+            for _ in range(3):
+                cn.matvec_noalloc(W, n_blocks, x, s)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free0
+            assert torch.cuda.memory_allocated() == held0
+            if timed:                                    # and its launches are not booked on the forward kernel's account
+                assert cn.profile_read(cn.KERNEL_FORWARD)[1] == before
+        finally:
+            cn.profile_enable(False)
+    ref = W.double().cpu().numpy() @ x.double().cpu().numpy().ravel()
+    assert np.max(np.abs(s.cpu().numpy() - ref)) / np.max(np.abs(ref)) <= 1e-5
