@@ -257,6 +257,18 @@ int codenet_decode_weights(const codenet_layer_t* layer, void* W_dev_out, codene
  * Section "Update stage on a single layer").  max_rel_dev: one float. */
 int codenet_check_invariance(const codenet_layer_t* layer, float* max_rel_dev, codenet_stream_t stream);
 
+/* Conditioning of the erasure decoding of one direction's code (Section "Some Notations": any a of the b columns of
+ * a systematic MDS generator are independent; "Decoding Algorithm", Appendix B: located outputs are solved from the
+ * others).  phase = CODENET_PHASE_FWD looks at G_r = [I | P_row], CODENET_PHASE_BWD at G_c.  Over every square
+ * sub-system A = P[F, Q]^T of s <= r located data outputs F and s parities Q: out[0] = the worst
+ * ||A||_inf ||A^-1||_inf, out[1] = the worst ||A^-1||_inf, out[2] = the worst factor by which errors of the node
+ * outputs can grow in a decoded output, max_a sum_b |A^-1[a,b]| (1 + sum_{k not in F} |P[k, Q_b]|).  `out` is host
+ * memory; nothing runs on the device.  A code without parity gives zeros; a singular sub-system gives infinity:
+ * such a generator is not MDS (two all-ones parities, a zero entry), the patterns that need the singular system are
+ * reported as uncorrectable when they occur, and a caller that wants every pattern of r located outputs decoded
+ * draws another generator.  Errors: BADARG. */
+int codenet_code_conditioning(const codenet_layer_t* layer, int phase, double out[3]);
+
 /* Copy one stored coded block (i, j) out as b_r x b_c floats (diagnostics / tests).
  * Errors: BADARG when the grid has no node at (i, j). */
 int codenet_get_block(const codenet_layer_t* layer, int i, int j, float* out_dev, codenet_stream_t stream);
@@ -288,6 +300,23 @@ int codenet_layer_dims(const codenet_layer_t* layer, int32_t dims[10]);
  * n = n_blocks, no parities and locate_mode OFF. */
 int codenet_matvec_noalloc(const float* W_dev, int rows, int cols, int n_blocks, const float* x_dev,
                            float* s_dev, codenet_stream_t stream);
+
+/* Bounded waits.  Every wait inside a kernel (a pipeline barrier of the tensor-core kernels) gives up after a time
+ * limit: the kernel then sets a flag of the layer, releases what it holds and returns, and every report written for
+ * the layer from then on carries CODENET_TIMEOUT instead of the outcome of its checks (the products of that launch
+ * are not valid) until codenet_reset_timeout acknowledges it.  The paper has no counterpart (its nodes are
+ * processes; a stuck one is found by the verification steps of Section "Decentralized Implementation").
+ *   codenet_set_wait_limit       the limit in nanoseconds for all later launches on this device (0: the default,
+ *                                about one second).
+ *   codenet_withhold_tile_loads  diagnostic: while on, the forward product kernel for batches >= 64 issues none of
+ *                                its tile loads, so the waits that depend on them run out after the limit.  Nothing
+ *                                faults and nothing is left in flight; it exists so that the give-up path can be
+ *                                exercised.
+ *   codenet_reset_timeout        clears the layer's flag.
+ * All three are asynchronous on `stream` and ordered with the launches on it.  Errors: BADARG, CUDA. */
+int codenet_set_wait_limit(uint64_t nanoseconds, codenet_stream_t stream);
+int codenet_withhold_tile_loads(int on, codenet_stream_t stream);
+int codenet_reset_timeout(codenet_layer_t* layer, codenet_stream_t stream);
 
 /* Kernels launched by this library since it was loaded (all streams). */
 uint64_t codenet_launch_count(void);

@@ -507,6 +507,59 @@ static int invert_small(int s, const double* A, double* inv) {
   return 1;
 }
 
+/* Conditioning of the erasure decoding of one direction's code (Section "Some Notations": any a of the b columns
+ * of the generator are independent; "Decoding Algorithm": located outputs are solved from the remaining ones).
+ * Every erasure sub-system is a square matrix A = P[F, Q]^T, F a set of s data indices, Q a set of s parity
+ * indices, 1 <= s <= r.  out[0] = worst ||A||_inf ||A^-1||_inf, out[1] = worst ||A^-1||_inf, out[2] = worst
+ * amplification of node-output errors into a decoded output,
+ *   max_a sum_b |A^-1[a, b]| (1 + sum_{k not in F} |P[k, Q_b]|);
+ * a singular sub-system gives infinity. */
+static void conditioning_rec(const double* P, int kd, int r, int s, int* F, int nF, int startF, double* out) {
+  if (nF < s) {
+    for (int k = startF; k < kd; ++k) { F[nF] = k; conditioning_rec(P, kd, r, s, F, nF + 1, k + 1, out); }
+    return;
+  }
+  /* every choice of s parities: bit masks with s bits */
+  for (unsigned mask = 0; mask < (1u << r); ++mask) {
+    int Q[8], nQ = 0;
+    for (int q = 0; q < r; ++q) if ((mask >> q) & 1u) Q[nQ++] = q;
+    if (nQ != s) continue;
+    double A[64], Ai[64];
+    for (int a = 0; a < s; ++a)
+      for (int b = 0; b < s; ++b) A[a * s + b] = P[F[b] * r + Q[a]];
+    if (!invert_small(s, A, Ai)) { out[0] = out[1] = out[2] = INFINITY; continue; }
+    double nA = 0.0, nAi = 0.0, amp = 0.0;
+    for (int a = 0; a < s; ++a) {
+      double ra = 0.0, ri = 0.0, am = 0.0;
+      for (int b = 0; b < s; ++b) {
+        ra += fabs(A[a * s + b]);
+        ri += fabs(Ai[a * s + b]);
+        double w = 1.0;
+        for (int k = 0; k < kd; ++k) {
+          int inF = 0;
+          for (int f = 0; f < s; ++f) if (F[f] == k) inF = 1;
+          if (!inF) w += fabs(P[k * r + Q[b]]);
+        }
+        am += fabs(Ai[a * s + b]) * w;
+      }
+      if (ra > nA) nA = ra;
+      if (ri > nAi) nAi = ri;
+      if (am > amp) amp = am;
+    }
+    if (nA * nAi > out[0]) out[0] = nA * nAi;
+    if (nAi > out[1]) out[1] = nAi;
+    if (amp > out[2]) out[2] = amp;
+  }
+}
+
+void orc_code_conditioning(const orc_layer_t* L, int phase, double out[3]) {
+  int n_cw, K, kd, r, len; const double* P;
+  phase_geometry(L, phase, &n_cw, &K, &kd, &r, &len, &P);
+  out[0] = out[1] = out[2] = 0.0;
+  int F[8];
+  for (int s = 1; s <= r && s <= kd && s <= 8; ++s) conditioning_rec(P, kd, r, s, F, 0, 0, out);
+}
+
 /* Column k of the parity-check matrix H = [P^T | -I]  (r entries). */
 static void h_column(const double* P, int kd, int r, int k, double* col) {
   for (int q = 0; q < r; ++q) col[q] = k < kd ? P[k * r + q] : (k - kd == q ? -1.0 : 0.0);

@@ -124,6 +124,10 @@ void orc_backward_update(orc_layer_t* L, const float* Delta, const float* X, int
 
 void orc_decode_weights(const orc_layer_t* L, float* W_out /* n_out x n_in */);
 double orc_check_invariance(const orc_layer_t* L);
+/* Conditioning of the erasure decoding of the code of one direction (phase 0: G_r, phase 1: G_c), over every square
+ * sub-system of the parity part with at most r unknowns: out[0] worst ||A||_inf ||A^-1||_inf, out[1] worst
+ * ||A^-1||_inf, out[2] worst amplification of node-output errors into a decoded output. */
+void orc_code_conditioning(const orc_layer_t* L, int phase, double out[3]);
 
 orc_net_t* orc_net_create(orc_layer_t** layers, int L, int activation, int loss);
 void orc_net_free(orc_net_t* net);

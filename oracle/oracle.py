@@ -107,6 +107,8 @@ def lib():
     L.orc_backward_update.argtypes = [vp, fp, fp, C.c_int, C.c_float, C.POINTER(Fault),
                                       C.c_uint32, fp, C.POINTER(Report)]
     L.orc_decode_weights.argtypes = [vp, fp]
+    L.orc_code_conditioning.argtypes = [vp, C.c_int, C.POINTER(C.c_double)]
+    L.orc_code_conditioning.restype = None
     L.orc_check_invariance.argtypes = [vp]
     L.orc_check_invariance.restype = C.c_double
     L.orc_net_create.argtypes = [C.POINTER(vp), C.c_int, C.c_int, C.c_int]
@@ -309,6 +311,12 @@ class Layer:
         W = np.empty((self.n_out, self.n_in), np.float32)
         lib().orc_decode_weights(self.h, _fp(W))
         return W
+
+    def code_conditioning(self, phase):
+        """(worst condition number, worst ||A^-1||, worst error amplification) over the erasure sub-systems."""
+        out = (C.c_double * 3)()
+        lib().orc_code_conditioning(self.h, phase, out)
+        return float(out[0]), float(out[1]), float(out[2])
 
     def check_invariance(self):
         return float(lib().orc_check_invariance(self.h))

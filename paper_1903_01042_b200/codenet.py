@@ -98,6 +98,14 @@ def lib():
     L.codenet_get_block.argtypes = [vp, ip, ip, vp, vp]
     L.codenet_get_checksums.argtypes = [vp, ip, ip, vp, vp, vp]
     L.codenet_layer_dims.argtypes = [vp, C.POINTER(C.c_int32)]
+    L.codenet_code_conditioning.argtypes = [vp, ip, C.POINTER(C.c_double)]
+    L.codenet_code_conditioning.restype = ip
+    L.codenet_set_wait_limit.argtypes = [C.c_uint64, vp]
+    L.codenet_set_wait_limit.restype = ip
+    L.codenet_withhold_tile_loads.argtypes = [ip, vp]
+    L.codenet_withhold_tile_loads.restype = ip
+    L.codenet_reset_timeout.argtypes = [vp, vp]
+    L.codenet_reset_timeout.restype = ip
     L.codenet_free_layer.argtypes = [vp]
     L.codenet_free_layer.restype = None
     L.codenet_free_net.argtypes = [vp]
@@ -347,6 +355,25 @@ def decode_weights(layer, out=None):
         out = torch.empty((layer.n_out, layer.n_in), dtype=dt, device="cuda")
     _check(lib().codenet_decode_weights(layer.h, _ptr(out), _stream()))
     return out
+
+
+def code_conditioning(layer, phase):
+    """codenet_code_conditioning: (worst condition number, worst ||A^-1||, worst error amplification)."""
+    out = (C.c_double * 3)()
+    _check(lib().codenet_code_conditioning(layer.h, int(phase), out))
+    return float(out[0]), float(out[1]), float(out[2])
+
+
+def set_wait_limit(nanoseconds):
+    _check(lib().codenet_set_wait_limit(int(nanoseconds), _stream()))
+
+
+def withhold_tile_loads(on):
+    _check(lib().codenet_withhold_tile_loads(1 if on else 0, _stream()))
+
+
+def reset_timeout(layer):
+    _check(lib().codenet_reset_timeout(layer.h, _stream()))
 
 
 def check_invariance(layer):

@@ -1,6 +1,8 @@
 // C interface of libcodenet: argument checks, layout planning, workspace, launch order.
 #include "codenet_internal.cuh"
 
+#include <algorithm>
+#include <cmath>
 #include <new>
 #include <vector>
 
@@ -89,7 +91,79 @@ void profile_end(int kernel, cudaStream_t st) {
 }
 }  // namespace codenet
 
+namespace {
+// Inverse of an s x s matrix (s <= CODENET_MAX_PARITY) by elimination with partial pivoting; false when singular.
+bool host_invert(int s, const double* A, double* inv) {
+  double a[CODENET_MAX_PARITY][2 * CODENET_MAX_PARITY];
+  for (int r = 0; r < s; ++r)
+    for (int c = 0; c < s; ++c) { a[r][c] = A[r * s + c]; a[r][s + c] = r == c ? 1.0 : 0.0; }
+  for (int pv = 0; pv < s; ++pv) {
+    int best = pv;
+    for (int r = pv + 1; r < s; ++r) if (std::fabs(a[r][pv]) > std::fabs(a[best][pv])) best = r;
+    if (a[best][pv] == 0.0) return false;
+    for (int c = 0; c < 2 * s; ++c) std::swap(a[pv][c], a[best][c]);
+    const double piv = a[pv][pv];
+    for (int c = 0; c < 2 * s; ++c) a[pv][c] /= piv;
+    for (int r = 0; r < s; ++r) {
+      if (r == pv) continue;
+      const double f = a[r][pv];
+      for (int c = 0; c < 2 * s; ++c) a[r][c] -= f * a[pv][c];
+    }
+  }
+  for (int r = 0; r < s; ++r) for (int c = 0; c < s; ++c) inv[r * s + c] = a[r][s + c];
+  return true;
+}
+
+// Worst figures over every erasure sub-system of the parity part P (k x r): see codenet_code_conditioning.
+void code_conditioning(const std::vector<float>& P, int k, int r, double out[3]) {
+  out[0] = out[1] = out[2] = 0.0;
+  for (int s = 1; s <= r && s <= k; ++s) {
+    std::vector<int> F(s);
+    for (int a = 0; a < s; ++a) F[a] = a;
+    for (;;) {
+      for (unsigned mask = 0; mask < (1u << r); ++mask) {
+        int Q[CODENET_MAX_PARITY], nq = 0;
+        for (int q = 0; q < r; ++q) if ((mask >> q) & 1u) Q[nq++] = q;
+        if (nq != s) continue;
+        double A[CODENET_MAX_PARITY * CODENET_MAX_PARITY], Ai[CODENET_MAX_PARITY * CODENET_MAX_PARITY];
+        for (int a = 0; a < s; ++a) for (int b = 0; b < s; ++b) A[a * s + b] = (double)P[(size_t)F[b] * r + Q[a]];
+        if (!host_invert(s, A, Ai)) { out[0] = out[1] = out[2] = INFINITY; continue; }
+        double w[CODENET_MAX_PARITY];
+        for (int b = 0; b < s; ++b) {
+          w[b] = 1.0;
+          for (int kk = 0; kk < k; ++kk) {
+            bool in_f = false;
+            for (int f = 0; f < s; ++f) in_f = in_f || F[f] == kk;
+            if (!in_f) w[b] += std::fabs((double)P[(size_t)kk * r + Q[b]]);
+          }
+        }
+        double na = 0.0, ni = 0.0, amp = 0.0;
+        for (int a = 0; a < s; ++a) {
+          double ra = 0.0, ri = 0.0, am = 0.0;
+          for (int b = 0; b < s; ++b) { ra += std::fabs(A[a * s + b]); ri += std::fabs(Ai[a * s + b]); am += std::fabs(Ai[a * s + b]) * w[b]; }
+          na = std::max(na, ra); ni = std::max(ni, ri); amp = std::max(amp, am);
+        }
+        out[0] = std::max(out[0], na * ni); out[1] = std::max(out[1], ni); out[2] = std::max(out[2], amp);
+      }
+      // next combination of s data indices out of k
+      int pos = s - 1;
+      while (pos >= 0 && F[pos] == k - s + pos) --pos;
+      if (pos < 0) break;
+      ++F[pos];
+      for (int a = pos + 1; a < s; ++a) F[a] = F[a - 1] + 1;
+    }
+  }
+}
+}  // namespace
+
 extern "C" {
+
+int codenet_code_conditioning(const codenet_layer_t* L, int phase, double out[3]) {
+  if (!L || !out || (phase != CODENET_PHASE_FWD && phase != CODENET_PHASE_BWD)) return CODENET_E_BADARG;
+  if (phase == CODENET_PHASE_FWD) code_conditioning(L->P_row_host, L->g.m, L->g.r_row, out);
+  else code_conditioning(L->P_col_host, L->g.n, L->g.r_col, out);
+  return CODENET_OK;
+}
 
 int codenet_profile_enable(int on) {
   g_prof.on = on != 0;

@@ -27,7 +27,11 @@ constexpr int TC_THREADS = 192;          // warp 0: TMA producer, warp 1: MMA is
 constexpr int TC_TILE_M = 128;
 constexpr int TC_KBYTES = 128;           // one 128-byte swizzle atom of K per stage
 constexpr uint32_t TC_SPIN_LIMIT = 1u << 24;
-constexpr unsigned long long TC_WAIT_NS = 1000000000ull;   // a stuck wait gives up after about a second
+// How long a stuck wait keeps trying before it gives up (codenet_set_wait_limit; about a second unless set), and a
+// diagnostic switch: the producer warp of the forward product kernel issues no tile loads at all, so that the waits
+// that depend on them run out (codenet_withhold_tile_loads: exercises the give-up path without any fault).
+__constant__ unsigned long long c_wait_ns = 1000000000ull;
+__constant__ int c_withhold_loads = 0;
 
 // ---- PTX wrappers -----------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -60,7 +64,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
     if ((spin & 1023u) == 1023u) {
       const unsigned long long now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > TC_WAIT_NS) return false;
+      else if (now - t0 > c_wait_ns) return false;
     }
   }
   return false;
@@ -200,7 +204,7 @@ tc_products_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_consta
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----
-    for (int k = 0; k < p.ksteps; ++k) {
+    for (int k = 0; k < (c_withhold_loads ? 0 : p.ksteps); ++k) {
       const int s = k % STAGES;
       if (k >= STAGES && !mbar_wait(&empty[s], ((k / STAGES) - 1) & 1)) { s_fail = 1; break; }
       mbar_expect_tx(&full[s], a_bytes + b_bytes);
@@ -250,9 +254,10 @@ tc_products_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_consta
     tc_commit(&accum_full);   // arrives when every instruction issued above has completed
   } else if (warp >= 2) {
     // ---- epilogue: tensor memory -> registers -> Y ----
-    const bool ok = mbar_wait(&accum_full, 0);
+    bool ok = mbar_wait(&accum_full, 0);
     if (!ok) s_fail = 1;
     tc_fence_after();
+    if (*reinterpret_cast<volatile int*>(&s_fail)) ok = false;   // the multiplication gave up: nothing to read back
     const int quad = warp & 3;                   // the lane quadrant this warp may read
     if (ok) {
       for (int tc = 0; tc < MT * N; tc += 32) {
@@ -1212,3 +1217,26 @@ cudaError_t launch_tc_backward_update(const codenet_layer_impl& L, int B, float 
 }
 
 }  // namespace codenet
+
+// ---- bounded waits: limit, diagnostic switch, acknowledgement -------------------------------------------------
+extern "C" {
+
+int codenet_set_wait_limit(uint64_t nanoseconds, codenet_stream_t stream) {
+  const unsigned long long v = nanoseconds ? (unsigned long long)nanoseconds : 1000000000ull;
+  return cudaMemcpyToSymbolAsync(codenet::c_wait_ns, &v, sizeof(v), 0, cudaMemcpyHostToDevice,
+                                 reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? CODENET_OK : CODENET_E_CUDA;
+}
+
+int codenet_withhold_tile_loads(int on, codenet_stream_t stream) {
+  const int v = on ? 1 : 0;
+  return cudaMemcpyToSymbolAsync(codenet::c_withhold_loads, &v, sizeof(v), 0, cudaMemcpyHostToDevice,
+                                 reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess ? CODENET_OK : CODENET_E_CUDA;
+}
+
+int codenet_reset_timeout(codenet_layer_t* layer, codenet_stream_t stream) {
+  if (!layer) return CODENET_E_BADARG;
+  return cudaMemsetAsync(layer->ws.tc_flag, 0, sizeof(int), reinterpret_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? CODENET_OK : CODENET_E_CUDA;
+}
+
+}  // extern "C"

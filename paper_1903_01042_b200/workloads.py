@@ -51,9 +51,35 @@ def labels(batch, n_classes, seed=0, iteration=0):
     return _rng(seed, 900000 + iteration).integers(0, n_classes, size=(batch,), dtype=np.int32)
 
 
+COND_LIMIT = 1e3   # a drawn generator is kept when every erasure sub-system is better conditioned than this
+
+
+def worst_condition(P):
+    """Largest ||A||_inf ||A^-1||_inf over the square sub-systems A = P[F, Q]^T of a parity part P (k x r): the
+    systems erasure decoding solves when the data outputs F are located and the parities Q are used."""
+    import itertools
+    P = np.asarray(P, np.float64)
+    k, r = P.shape
+    worst = 0.0
+    for s in range(1, min(k, r) + 1):
+        for F in itertools.combinations(range(k), s):
+            for Q in itertools.combinations(range(r), s):
+                A = P[np.ix_(F, Q)].T
+                if abs(np.linalg.det(A)) == 0.0:
+                    return float("inf")
+                worst = max(worst, float(np.abs(A).sum(1).max() * np.abs(np.linalg.inv(A)).sum(1).max()))
+    return worst
+
+
 def gaussian_parity(k, r, seed=0, which=0):
-    """Parity part P (k x r) of a systematic real generator [I | P], entries N(0, 1)."""
-    return _rng(seed, 7000 + which).standard_normal((k, r)).astype(np.float32)
+    """Parity part P (k x r) of a systematic real generator [I | P], entries N(0, 1).  A draw with an erasure
+    sub-system worse conditioned than COND_LIMIT is thrown away and the next stream of the same seed is drawn
+    (a Gaussian matrix is MDS with probability one, but a draw can come arbitrarily close to a singular minor)."""
+    for attempt in range(64):
+        P = _rng(seed, 7000 + which + 100000 * attempt).standard_normal((k, r)).astype(np.float32)
+        if r == 0 or worst_condition(P) <= COND_LIMIT:
+            return P
+    raise RuntimeError("no well-conditioned generator found")
 
 
 def check_slice(length, slices=8):

@@ -196,6 +196,8 @@ def _injected_faults_decisions(cn, orc, shape, B, iterations, locate_mode=2):
         # outputs by the conditioning of the erasure system; checksum codes (all-ones P) do not
         tol_f = TOL_F32 if (not gauss or rf.status == cn.CLEAN) else TOL_DECODED
         tol_b = TOL_F32 if (not gauss or rb.status == cn.CLEAN) else TOL_DECODED
+        if gauss:   # the looser bar stays inside what the conditioning of this code can amplify
+            assert TOL_DECODED <= max(p.o.code_conditioning(0)[2], p.o.code_conditioning(1)[2]) * TOL_F32
         assert _rel(S.cpu().numpy(), So) <= tol_f
         assert _rel(Cg.cpu().numpy(), Co) <= tol_b
         seen.add(rf.status)
@@ -293,6 +295,57 @@ def test_joint_location_of_up_to_r_minus_1_nodes(cn, orc, phase, r, B):
             assert _rel(Yg.cpu().numpy(), Yo) <= TOL_DECODED
 
 
+def test_code_conditioning_matches_the_oracle_and_singular_generators_are_reported(cn, orc):
+    """The library's figures for the erasure sub-systems of both codes are the oracle's, and a generator with a
+    singular sub-system (a zero entry: the lone parity cannot rebuild that data output; two all-ones parities)
+    shows as infinite on both sides."""
+    for (m, n, rr, rc, seed) in [(4, 4, 2, 2, 1), (8, 8, 2, 2, 0), (3, 5, 3, 4, 4), (4, 4, 1, 1, None)]:
+        W = wl.weights(8 * m, 8 * n, seed=9)
+        Pr, Pc = (None, None) if seed is None else (wl.gaussian_parity(m, rr, seed, 0), wl.gaussian_parity(n, rc, seed, 1))
+        p = Pair(cn, orc, W, m, n, rr, rc, Pr, Pc)
+        for phase in (0, 1):
+            a, b = cn.code_conditioning(p.g, phase), p.o.code_conditioning(phase)
+            assert np.allclose(a, b, rtol=1e-12, atol=0.0), (m, n, rr, rc, phase, a, b)
+            assert a[0] <= wl.COND_LIMIT          # the generator the workloads draw passed the screen
+    bad = np.ones((4, 1), np.float32)
+    bad[2, 0] = 0.0
+    for (rr, Pr) in [(1, bad), (2, None)]:
+        p = Pair(cn, orc, wl.weights(32, 32, seed=9), 4, 4, rr, 1, Pr, None)
+        assert cn.code_conditioning(p.g, 0)[0] == float("inf") and p.o.code_conditioning(0)[0] == float("inf")
+        assert np.isfinite(cn.code_conditioning(p.g, 1)[0])
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_and_the_layer_recovers(cn, orc):
+    """A forward launch on tensor-core tiles whose producer warp is told to issue no tile loads: the waits that
+    depend on those loads give up after the (shortened) limit, the kernel releases its tensor memory and returns
+    by itself, and the report of the call says TIMEOUT.  Nothing faults and nothing stays in flight.  After the
+    acknowledgement the same layer runs normally again and agrees with the oracle."""
+    W = wl.weights(512, 512, seed=61)
+    p = Pair(cn, orc, W, 2, 2, 1, 1, batch_max=64, math=1)          # fp32 blocks, TF32 tiles, 256 x 256 blocks
+    X = wl.gaussian_inputs(64, 512, seed=62)
+    rep = cn.new_reports(1)
+    S = cn.forward(p.g, _dev(X), rep_dev=rep)                       # a normal launch first
+    So, ro = p.o.forward(X)
+    assert cn.read_reports(rep)[0].status == cn.CLEAN and _rel(S.cpu().numpy(), So) <= TOL_LOWP
+    try:
+        cn.set_wait_limit(2_000_000)                                # two milliseconds instead of about a second
+        cn.withhold_tile_loads(True)
+        cn.forward(p.g, _dev(X), rep_dev=rep)
+        cn.withhold_tile_loads(False)
+        torch.cuda.synchronize()                                    # the kernel came back by itself
+        assert cn.read_reports(rep)[0].status == cn.TIMEOUT
+        cn.forward(p.g, _dev(X), rep_dev=rep)                       # the flag stays until it is acknowledged
+        assert cn.read_reports(rep)[0].status == cn.TIMEOUT
+    finally:
+        cn.withhold_tile_loads(False)
+        cn.set_wait_limit(0)
+    cn.reset_timeout(p.g)
+    S = cn.forward(p.g, _dev(X), rep_dev=rep)
+    assert cn.read_reports(rep)[0].decisions() == ro.decisions()
+    assert cn.read_reports(rep)[0].status == cn.CLEAN
+    assert _rel(S.cpu().numpy(), So) <= TOL_LOWP
+
+
 def test_check_rows_slices(cn, orc):
     W = wl.weights(64, 32, seed=12)
     p = Pair(cn, orc, W, 2, 2, 1, 1, batch_max=2, check_rows=8, check_cols=4)
@@ -357,6 +410,11 @@ def _run_config(cn, orc, cfg, iterations, tol, weight_tol, p=None, check_every=1
                 tol_decoded=None, lookahead=False, math=0):
     pairs, gnet, onet = _build_net(cn, orc, cfg, math=math)
     L = len(pairs)
+    if tol_decoded is not None:
+        # an erasure-decoded output carries the deviations of the node outputs it is solved from, amplified by
+        # at most the factor the code's conditioning gives: the looser bar must lie inside that envelope
+        amplification = max(pr.o.code_conditioning(ph)[2] for pr in pairs for ph in (0, 1))
+        assert tol <= tol_decoded <= amplification * tol, (tol_decoded, amplification)
     mode = {"bernoulli": 1, "exactly_one": 2, "none": 0}[cfg.fault_mode]
     prob = cfg.p if p is None else p
     it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")

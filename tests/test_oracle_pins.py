@@ -566,9 +566,136 @@ def test_step_matches_autograd_sgd(orc, loss_kind):
         assert all(r.status == orc.CLEAN for r in reps)
 
 
+def test_code_conditioning_closed_forms_and_brute_force(orc):
+    """Conditioning of the erasure sub-systems: closed forms for the all-ones checksum code and for the
+    generators of the paper's worked example, and an independent enumeration with numpy's inverse for seeded
+    Gaussian codes."""
+    import itertools
+    from paper_1903_01042_b200 import workloads as wl
+    W = np.zeros((12, 20), np.float32)
+    # all-ones single parity over k data outputs: A = [1]; a decoded output is parity minus the k - 1 others
+    lay = orc.Layer(W, 4, 5, 1, 1)
+    assert lay.code_conditioning(0) == (1.0, 1.0, 4.0) and lay.code_conditioning(1) == (1.0, 1.0, 5.0)
+    # the worked example: P_r = [[1, 1], [1, -1]], P_c = [[1, 1], [1, 2]]
+    toy = orc.Layer(np.zeros((4, 4), np.float32), 2, 2, 2, 2, P_row=[[1, 1], [1, -1]], P_col=[[1, 1], [1, 2]])
+    assert toy.code_conditioning(0) == (2.0, 1.0, 2.0)
+    # P_c: 1 x 1 systems 1 / |p| <= 1, amplification (1 + other) / |p| <= 3; the 2 x 2 system has inverse [[2, -1], [-1, 1]]
+    assert np.allclose(toy.code_conditioning(1), (3.0 * 3.0, 3.0, 3.0))
+    for (k, r, seed) in [(5, 2, 0), (6, 3, 4), (4, 4, 2)]:
+        P = wl.gaussian_parity(k, r, seed, 0)
+        lay = orc.Layer(np.zeros((2 * k, 8), np.float32), k, 2, r, 0, P_row=P)
+        worst = [0.0, 0.0, 0.0]
+        P64 = P.astype(np.float64)
+        for s in range(1, r + 1):
+            for F in itertools.combinations(range(k), s):
+                rest = [x for x in range(k) if x not in F]
+                for Q in itertools.combinations(range(r), s):
+                    A = P64[np.ix_(F, Q)].T
+                    Ai = np.linalg.inv(A)
+                    w = 1.0 + np.abs(P64[np.ix_(rest, Q)]).sum(axis=0)
+                    worst[0] = max(worst[0], np.abs(A).sum(1).max() * np.abs(Ai).sum(1).max())
+                    worst[1] = max(worst[1], np.abs(Ai).sum(1).max())
+                    worst[2] = max(worst[2], (np.abs(Ai) @ w).max())
+        assert np.allclose(lay.code_conditioning(0), worst, rtol=1e-10)
+        assert np.isclose(worst[0], wl.worst_condition(P), rtol=1e-10) and worst[0] <= wl.COND_LIMIT
+        assert lay.code_conditioning(1) == (0.0, 0.0, 0.0)      # no parity in that direction
+
+
+def test_node_check_threshold_has_a_rounding_floor_for_cancelling_checksums(orc):
+    """Blocks whose rows cancel exactly (every column sums to zero) have zero inner checksums u, so the
+    checksum-side scale of the node-check threshold, tau_rel * sum|u||x|, is zero, while the sum of the stored
+    (rounded) block outputs is a rounding residue of the order of 1e-7 * sum|y|.  The threshold's second term,
+    (tau_rel / 512) * sum|y|, is what keeps such a fault-free node from being flagged: without it this test
+    fails (the ratio is the residue over tau_abs = 1e-20).  The margin of the clean outputs stays below 0.1, and a
+    hit node is still found with its margin above 10."""
+    rng = np.random.default_rng(5)
+    m = n = 2
+    b = 48
+    W = np.zeros((m * b, n * b), np.float32)
+    for i in range(m):
+        for j in range(n):
+            a = np.round(rng.uniform(-1, 1, (b // 3, b)) * 1024) / 1024          # ten fractional bits: sums are exact
+            c = np.round(rng.uniform(-1, 1, (b // 3, b)) * 1024) / 1024
+            blk = np.concatenate([a, c, -(a + c)]).astype(np.float32)
+            assert np.all(blk.astype(np.float64).sum(axis=0) == 0.0)
+            W[i * b:(i + 1) * b, j * b:(j + 1) * b] = blk
+    lay = orc.Layer(W, m, n, 1, 1, tau_rel=1e-3, tau_abs=1e-20)
+    assert all(np.all(lay.u(i, j) == 0.0) for i in range(m + 1) for j in range(n))   # the checksums do cancel
+    worst = 0.0
+    for trial in range(20):
+        X = rng.standard_normal((3, n * b)).astype(np.float32)
+        S, rep = lay.forward(X)
+        Y = lay.forward_products(X)
+        assert np.any(Y.astype(np.float64).reshape(n, m + 1, b, 3).sum(axis=2) != 0.0)    # there is a residue to survive
+        assert rep.status == orc.CLEAN and rep.n_detected_cw == 0, trial
+        worst = max(worst, rep.max_margin_clean)
+    assert 0.0 < worst < 0.1
+    f = orc.make_fault(seed=2, mode=orc.FAULT_EXACTLY_ONE, sigma=10.0)
+    for it in range(10):
+        S, rep = lay.forward(rng.standard_normal((3, n * b)).astype(np.float32), f, it)
+        assert tuple(rep.flagged_mask) == tuple(rep.injected_mask)
+        assert rep.min_margin_hit > 10.0
+
+
 # ---------------------------------------------------------------------------------------------
 # bfloat16 storage
 # ---------------------------------------------------------------------------------------------
+
+def _bf16_rne_by_integers(x):
+    """Round-to-nearest-even of float32 values to bfloat16 (returned as float32), in integer arithmetic on the bit
+    patterns: keep the upper 16 bits, round up when the lower 16 are above half, or exactly half with an odd keeper."""
+    u = np.asarray(x, np.float32).view(np.uint32).astype(np.uint64)
+    low, keep = u & 0xFFFF, u >> 16
+    up = (low > 0x8000) | ((low == 0x8000) & ((keep & 1) == 1))
+    return ((keep + up.astype(np.uint64)) << 16).astype(np.uint32).view(np.float32)
+
+
+def test_bf16_storage_rounds_to_nearest_even_in_parity_blocks_and_updates(orc):
+    """The storage rounding of the oracle is round-to-nearest-even: pinned on sums that land exactly half-way
+    between two bfloat16 values (even and odd keepers), just above and just below half-way, against two
+    independent roundings (integer arithmetic on the bits; torch's float32 -> bfloat16 conversion).  Truncation,
+    or rounding half away from zero, fails the tie cases."""
+    import torch
+    m = n = 2
+    b = 8                                            # 8 x 8 blocks
+    h = np.float32(2.0 ** -8)                        # half a bfloat16 step at 1.0
+    # data blocks (all representable in bfloat16); the parity block-row holds W_0j + W_1j
+    base = np.array([1.0, 1.0078125, -1.0, -1.0078125, 1.5, 2.0, 0.75, 1.0], np.float32)
+    add = np.array([h, h, -h, -h, h * np.float32(1.5), h, h * np.float32(0.25), np.float32(2.0 ** -9)], np.float32)
+    assert np.array_equal(base, _bf16_rne_by_integers(base)) and np.array_equal(add, _bf16_rne_by_integers(add))
+    W = np.zeros((m * b, n * b), np.float32)
+    for c in range(n * b):
+        W[:b, c] = np.roll(base, c)
+        W[b:, c] = np.roll(add, c)
+    lay = orc.Layer(W, m, n, 1, 1, store_bf16=True, tau_rel=3e-2)
+    for j in range(n):
+        exact = (W[:b, j * b:(j + 1) * b].astype(np.float64) + W[b:, j * b:(j + 1) * b].astype(np.float64)).astype(np.float32)
+        want = _bf16_rne_by_integers(exact)
+        assert np.array_equal(want, torch.tensor(exact).to(torch.bfloat16).float().numpy())
+        got = lay.block(m, j)                        # parity block-row m, block-column j
+        assert np.array_equal(got, want), j
+        # the cases really are what they claim: ties that round down to an even keeper, ties that round up,
+        # and values a truncation would get wrong
+        trunc = (exact.view(np.uint32) & np.uint32(0xFFFF0000)).view(np.float32)
+        assert np.any(want != trunc) and np.any((exact.view(np.uint32) & 0xFFFF) == 0x8000)
+    # the coded update rounds once, from the exact sum, to nearest even as well
+    lr = 1.0
+    D = np.zeros((1, m * b), np.float32); D[0, :] = 1.0
+    X = np.zeros((1, n * b), np.float32); X[0, :] = np.tile(np.array([h, -h, h * np.float32(3.0), np.float32(2.0 ** -9)], np.float32), n * b // 4)
+    before = [[lay.block(i, j).astype(np.float64) if not (i == m and j == n) else None for j in range(n + 1)]
+              for i in range(m + 1)]
+    lay.update(D, X, lr)
+    Dt = np.concatenate([D[0, :b], D[0, b:], D[0, :b] + D[0, b:]])            # delta~ per block-row (all-ones code)
+    Xt = np.concatenate([X[0, :b], X[0, b:], X[0, :b] + X[0, b:]])            # x~ per block-column
+    for i in range(m + 1):
+        for j in range(n + 1):
+            if i == m and j == n:
+                continue
+            exact = (before[i][j] + lr * np.outer(Dt[i * b:(i + 1) * b], Xt[j * b:(j + 1) * b])).astype(np.float32)
+            want = _bf16_rne_by_integers(exact)
+            assert np.array_equal(want, torch.tensor(exact).to(torch.bfloat16).float().numpy())
+            assert np.array_equal(lay.block(i, j), want), (i, j)
+
 
 def test_bf16_storage_rounds_blocks_and_keeps_products_close(orc):
     from paper_1903_01042_b200 import workloads as wl
