@@ -582,6 +582,86 @@ def test_tensor_core_tiles_on_other_batches(cn, orc, name, math, batch):
     assert stats["detected"] > 0
 
 
+def test_config4_scaled_200_iterations_on_tensor_core_tiles(cn, orc):
+    """The iteration count configuration 4 names, at 2048 x 2048 (same grid, code, batch and error rate): decisions
+    as the oracle's at every checked step, weights inside the bfloat16 bound after all 200."""
+    cfg = wl.config("c4", scale=8)
+    stats = _run_config(cn, orc, cfg, 200, TOL_LOWP, 2e-3, weight_norm="fro", tol_decoded=3e-2, math=2, check_every=8)
+    assert stats["detected"] > 0 and stats["corrected"] > 0
+
+
+def test_config5_scaled_100_iterations_on_tensor_core_tiles(cn, orc):
+    """Configuration 5 at a quarter of its widths (nine layers, TF32 tiles, batch 64), 100 iterations at the largest
+    error rate of its sweep.  Every layer's TF32 products deviate by up to 2e-3 and the deviations add up through
+    the layers; the weights take lr times the deviation of delta per step."""
+    cfg = wl.config("c5", scale=4)
+    stats = _run_config(cn, orc, cfg, 100, TOL_LOWP * len(cfg.layers), 1e-3, p=1e-2, math=1, check_every=5)
+    assert stats["detected"] > 0
+
+
+def test_config2_2000_iterations_at_its_own_error_rate(cn, orc):
+    """Configuration 2 at the error rate it names (1e-3 per node and phase), 2000 of its iterations.  Decisions are
+    the oracle's at every step of the run.  Values: outputs within 1e-5 and weights within 1e-4 at every step until
+    the two runs part at a ReLU unit, which must not happen in the first 100 steps (the bar of the configuration).
+    Float against double evaluate a pre-activation s = W x a few 1e-7 apart; when an s falls between them, one side
+    sees f'(s) = 1 where the other sees 0, that unit's delta is dropped on one side only, and ONE row of one
+    layer's weights moves by lr * delta * x on one side only.  The test recognises exactly that signature (one
+    layer, one row) at the step where the weights part; any other first difference fails.  From then on the two
+    equally valid runs are compared on decisions only."""
+    cfg = wl.config("c2")
+    pairs, gnet, onet = _build_net(cn, orc, cfg)
+    L = len(pairs)
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fg = [cn.make_fault(seed=cfg.seed, layer=l, mode=1, p=cfg.p, sigma=cfg.sigma, iteration_dev=it_dev) for l in range(L)]
+    fo = [orc.make_fault(seed=cfg.seed, layer=l, mode=1, p=cfg.p, sigma=cfg.sigma) for l in range(L)]
+    reps = cn.new_reports(2 * L)
+    loss_dev = torch.zeros(1, device="cuda")
+    together, parted_at, detected = True, None, 0
+    for it in range(2000):
+        X, T = wl.layer_inputs(cfg, it)
+        it_dev.fill_(it)
+        cn.step(gnet, _dev(X), torch.tensor(T, device="cuda"), cfg.lr, faults=fg, reps_dev=reps, loss_dev=loss_dev)
+        lo, out_o, reps_o = onet.step(X, T, cfg.lr, fo, it)
+        rg = cn.read_reports(reps)
+        assert [r.decisions() for r in rg] == [r.decisions() for r in reps_o], it
+        detected += sum(r.n_detected_cw for r in rg)
+        if not together:
+            continue
+        assert _rel(gnet.output(1).cpu().numpy(), out_o) <= TOL_F32, it
+        devs = []
+        for pr in pairs:
+            wg, wo = cn.decode_weights(pr.g).float().cpu().numpy(), pr.o.decode_weights()
+            devs.append(np.max(np.abs(wg - wo), axis=1) / np.max(np.abs(wo)))
+        worst = [float(d.max()) for d in devs]
+        if max(worst) > 1e-5:
+            # the runs part here: one row of one layer, by about lr * delta * x, everything else as before
+            layers_off = [l for l in range(L) if worst[l] > 1e-5]
+            assert len(layers_off) == 1, (it, worst)
+            rows_off = np.flatnonzero(devs[layers_off[0]] > 1e-6)
+            assert len(rows_off) == 1 and worst[layers_off[0]] < 1e-2, (it, rows_off, worst)
+            together, parted_at = False, it
+    assert parted_at is None or parted_at > 100, parted_at
+    assert detected > 100
+
+
+def test_config4_full_size_iteration_against_the_oracle(cn, orc):
+    """One whole iteration of configuration 4 at full size (16384 x 16384 bfloat16, batch 128) compared with the
+    oracle element by element: decisions, outputs, loss, and every decoded weight."""
+    cfg = wl.config("c4")
+    stats = _run_config(cn, orc, cfg, 1, TOL_LOWP, 2e-3, p=2e-2, weight_norm="fro", tol_decoded=3e-2, math=2)
+    assert stats["detected"] > 0
+
+
+def test_config5_full_size_layers_against_the_oracle(cn, orc):
+    """Two whole iterations of the first two layers and the head of configuration 5 at full size (4096 x 4096,
+    batch 64, TF32 tiles) compared with the oracle element by element."""
+    import dataclasses
+    cfg = wl.config("c5")
+    cfg = dataclasses.replace(cfg, layers=cfg.layers[:2] + cfg.layers[-1:])
+    stats = _run_config(cn, orc, cfg, 2, TOL_LOWP * len(cfg.layers), 3e-4, p=2e-2, math=1)
+    assert stats["detected"] > 0
+
+
 @pytest.mark.parametrize("bf16,math", [(False, 1), (True, 2)])
 def test_tensor_core_update_moves_every_stored_block(cn, orc, bf16, math):
     """One step with a learning rate large enough for bfloat16 storage to see the update: every stored
