@@ -44,7 +44,9 @@ enum { CODENET_LOCATE_NONE = 0, CODENET_LOCATE_SYNDROME = 1, CODENET_LOCATE_NODE
 enum { CODENET_FAULT_NONE = 0, CODENET_FAULT_BERNOULLI = 1, CODENET_FAULT_EXACTLY_ONE = 2 };
 enum { CODENET_PHASE_FWD = 0, CODENET_PHASE_BWD = 1 };
 enum { CODENET_CLEAN = 0, CODENET_CORRECTED = 1, CODENET_FALLBACK = 2, CODENET_FAILED = 3,
-       CODENET_TIMEOUT = 4 };
+       CODENET_TIMEOUT = 4,
+       CODENET_DISAGREE = 5 /* a verification step found two evaluations that differ: restore the last checkpoint */ };
+enum { CODENET_PHASE_ENCODE = 2, CODENET_PHASE_INPUT = 3, CODENET_PHASE_CHECK = 4, CODENET_PHASE_DECODE = 5 };
 enum { CODENET_ACT_IDENTITY = 0, CODENET_ACT_RELU = 1 };
 enum { CODENET_LOSS_MSE_MEAN = 0, CODENET_LOSS_SOFTMAX_CE = 1 };
 
@@ -107,6 +109,32 @@ typedef struct {
   const uint32_t* iteration_dev;  /* DEVICE counter read by the kernels (lets a captured     */
                                   /* CUDA graph be replayed); NULL = iteration 0             */
 } codenet_fault_t;
+
+/* Soft errors in the steps around the products (Section "Decentralized Implementation": under Error Model 2 the
+ * additional encoding, the generation of a node's input sub-vector by the activation / post-multiplication step,
+ * the error detection and the decoding can err as well).  Unit u of small-step phase ph is hit in an iteration when
+ * word 0 of Philox4x32-10(counter = (iteration, u, 0, 0), key = (seed, layer << 8 | ph)) is below that phase's
+ * p_q32; noise values are drawn like those of codenet_fault_t with the same key.
+ *   CODENET_PHASE_ENCODE  drawn in the backward call: unit j for x~_j (j >= n), unit (n + r_col) + i for delta~_i
+ *                         (i >= m).  The whole encoded sub-vector is off by noise; the update (blocks and inner
+ *                         checksums alike) takes it as it is, so the stored parity blocks of that block-column /
+ *                         block-row leave the code and the next products on them show it.
+ *   CODENET_PHASE_INPUT   feedforward products: unit = node i * (n + r_col) + j.  The node's own copy of x_j is off
+ *                         by a noise vector nu, so its output is off by W~_ij nu; it counts among the injected nodes
+ *                         of the report.
+ *   CODENET_PHASE_CHECK   unit = phase of the call * 64 + codeword: one of the two evaluations of the codeword's
+ *                         parity checks is off by a noise value ("Errors in Error-Detection under Error Model 2").
+ *   CODENET_PHASE_DECODE  same units, detected codewords only: one of the two lists of nodes found erroneous has
+ *                         the membership of one node changed ("Errors in decoding under Error Model 2").
+ * The two verification steps compare the evaluations; a difference makes the report's status CODENET_DISAGREE and
+ * leaves the codeword as it is: the caller restores the last checkpoint (codenet_checkpoint_restore). */
+typedef struct {
+  uint32_t seed;
+  uint32_t layer;
+  uint32_t p_encode_q32, p_input_q32, p_check_q32, p_decode_q32;   /* floor(p * 2^32) per phase; 0 = never */
+  float sigma;
+  const uint32_t* iteration_dev;  /* DEVICE counter as in codenet_fault_t; NULL = iteration 0 */
+} codenet_small_faults_t;
 
 /* Written on the device by each call that checks outputs. */
 typedef struct {
@@ -198,6 +226,11 @@ int codenet_regenerate_block(codenet_layer_t* layer, int i, int j, int along, co
  * NOMEM (save could not allocate), CUDA. */
 int codenet_checkpoint_save(codenet_layer_t* layer, codenet_stream_t stream);
 int codenet_checkpoint_restore(codenet_layer_t* layer, codenet_stream_t stream);
+
+/* Plan for soft errors in the small steps of every later call on this layer (copied; NULL switches them off).  A plan
+ * with p_input_q32 > 0 makes the layer allocate one more buffer of the size of its node outputs; this call may
+ * therefore allocate and synchronise.  Errors: BADARG, NOMEM. */
+int codenet_layer_set_small_faults(codenet_layer_t* layer, const codenet_small_faults_t* plan);
 
 /* Stand-alone detection / location / erasure decoding ("General Error-Detection Method" and
  * "Decoding Algorithm", Appendix B) of un-reduced node outputs the caller supplies.

@@ -51,6 +51,9 @@ struct orc_layer {
   float** ck_blk; /* the last checkpoint (same shapes), NULL until one is taken */
   float** ck_u;
   float** ck_v;
+  orc_small_faults_t small;  /* soft errors in the small steps; all probabilities zero: none */
+  int have_small;
+  uint32_t small_iteration;  /* iteration of the call in progress (orc_forward / orc_backward_update set it) */
 };
 
 static float store_w(const orc_layer_t* L, double x) {
@@ -128,6 +131,22 @@ int orc_node_hit(const orc_fault_t* f, uint32_t phase, uint32_t iteration, uint3
     return (out[0] % n_active) == active_index;
   }
   return 0;
+}
+
+int orc_small_hit(const orc_small_faults_t* plan, uint32_t phase, uint32_t iteration, uint32_t unit) {
+  if (!plan) return 0;
+  const uint32_t p = phase == ORC_PHASE_ENCODE ? plan->p_encode_q32 : phase == ORC_PHASE_INPUT ? plan->p_input_q32
+                   : phase == ORC_PHASE_CHECK ? plan->p_check_q32 : plan->p_decode_q32;
+  if (p == 0) return 0;
+  uint32_t key[2] = {plan->seed, (plan->layer << 8) | phase};
+  uint32_t c[4] = {iteration, unit, 0u, 0u}, out[4];
+  orc_philox4x32_10(c, key, out);
+  return out[0] < p;
+}
+
+void orc_layer_set_small_faults(orc_layer_t* L, const orc_small_faults_t* plan) {
+  L->have_small = plan != NULL;
+  if (plan) L->small = *plan;
 }
 
 /* ------------------------------------------------------------------------------------------ */
@@ -351,6 +370,8 @@ int orc_regenerate_block(orc_layer_t* L, int i, int j, int along) {
     }
     dst[e] = store_w(L, acc);
   }
+  /* everything the node stored is generated again, its inner checksums included */
+  recompute_checksums(L, i, j);
   return 0;
 }
 
@@ -757,6 +778,18 @@ void orc_detect_decode(const orc_layer_t* L, int phase, float* Y, const float* V
       else if (ratio > rep->max_margin_clean) rep->max_margin_clean = ratio;
     }
     const int detected = (r > 0 && smax > tau_syn) || flags != 0;
+    /* Verification step of the error detection (Section "Decentralized Implementation", "Errors in Error-Detection
+     * under Error Model 2"): the evaluation of the codeword's parity checks is made twice and compared.  A soft error
+     * in one evaluation shifts its value by a noise sample; any difference means the nodes disagree, and the caller
+     * has to restore the last checkpoint (the codeword is left as it is). */
+    const uint32_t vunit = (uint32_t)(phase * 64 + cw);
+    if (L->have_small && orc_small_hit(&L->small, ORC_PHASE_CHECK, L->small_iteration, vunit)) {
+      const float shift = orc_noise(L->small.seed, L->small.layer, ORC_PHASE_CHECK, L->small_iteration, vunit, 0u, L->small.sigma);
+      if (shift != 0.0f) {
+        if (rep->status < ORC_DISAGREE) rep->status = ORC_DISAGREE;
+        continue;
+      }
+    }
     if (!detected) continue;
     rep->detected_mask |= (uint64_t)1 << cw;
     rep->n_detected_cw++;
@@ -770,6 +803,19 @@ void orc_detect_decode(const orc_layer_t* L, int phase, float* Y, const float* V
     }
     rep->flagged_mask[cw] = F;
     rep->n_flagged_nodes += (uint32_t)popcount64(F);
+    /* Verification step of the decoding ("Errors in decoding under Error Model 2"): the list of nodes found
+     * erroneous is made twice and compared.  A soft error in one evaluation changes the membership of one node
+     * (chosen by the generator); the lists then differ and the decoding is deemed erroneous. */
+    if (L->have_small && orc_small_hit(&L->small, ORC_PHASE_DECODE, L->small_iteration, vunit)) {
+      uint32_t key[2] = {L->small.seed, (L->small.layer << 8) | ORC_PHASE_DECODE};
+      uint32_t c[4] = {L->small_iteration, vunit, 1u, 0u}, o[4];
+      orc_philox4x32_10(c, key, o);
+      const uint64_t F_other = F ^ ((uint64_t)1 << (o[0] % (uint32_t)K));
+      if (F_other != F) {
+        if (rep->status < ORC_DISAGREE) rep->status = ORC_DISAGREE;
+        continue;
+      }
+    }
     if (ok && popcount64(F) > r) ok = 0;
 
     if (ok) {
@@ -835,7 +881,7 @@ void orc_detect_decode(const orc_layer_t* L, int phase, float* Y, const float* V
         memcpy(out, Yclean + (size_t)cw * K * n_el, (size_t)K * n_el * sizeof(float));
         if (rep->status < ORC_FALLBACK) rep->status = ORC_FALLBACK;
       } else {
-        rep->status = ORC_FAILED;
+        if (rep->status < ORC_FAILED) rep->status = ORC_FAILED;
       }
     }
   }
@@ -853,9 +899,33 @@ void orc_forward(orc_layer_t* L, const float* X, int B, const orc_fault_t* f,
   float* Y = (float*)malloc(total * sizeof(float));
   float* Yc = (float*)malloc(total * sizeof(float));
   uint64_t inj[64];
+  L->small_iteration = iteration;
   orc_forward_products(L, X, B, Y);
   memcpy(Yc, Y, total * sizeof(float));
   orc_inject(L, ORC_PHASE_FWD, f, iteration, Y, B, inj);
+  if (L->have_small && L->small.p_input_q32) {
+    /* a node whose own copy of x_j is off by a noise vector nu produces W~_ij (x_j + nu): its output is off by
+     * W~_ij nu, like any other erroneous output (and it counts among the injected nodes) */
+    const orc_small_faults_t* sf = &L->small;
+    const int bc = L->b_c;
+    double* nu = (double*)malloc((size_t)bc * B * sizeof(double));
+    for (int j = 0; j < n; ++j)
+      for (int i = 0; i < M; ++i) {
+        const uint32_t node = (uint32_t)(i * L->Nn + j);
+        if (!orc_small_hit(sf, ORC_PHASE_INPUT, iteration, node)) continue;
+        inj[j] |= (uint64_t)1 << i;
+        for (int e = 0; e < bc * B; ++e) nu[e] = (double)orc_noise(sf->seed, sf->layer, ORC_PHASE_INPUT, iteration, node, (uint32_t)e, sf->sigma);
+        const float* w = L->blk[i * L->Nn + j];
+        float* y = Y + ((size_t)(j * M + i) * br) * B;
+        for (int r = 0; r < br; ++r)
+          for (int b = 0; b < B; ++b) {
+            double acc = 0.0;
+            for (int c = 0; c < bc; ++c) acc += (double)w[(size_t)r * bc + c] * nu[(size_t)c * B + b];
+            y[(size_t)r * B + b] = (float)((double)y[(size_t)r * B + b] + acc);
+          }
+      }
+    free(nu);
+  }
   orc_detect_decode(L, ORC_PHASE_FWD, Y, X, B, Yc, inj, rep);
   /* s_i = sum_j y_ij (the row All-Reduce of the decentralised algorithm) */
   for (int b = 0; b < B; ++b)
@@ -872,12 +942,35 @@ void orc_forward(orc_layer_t* L, const float* X, int B, const orc_fault_t* f,
 
 /* Coded rank-B update (step O3, the three update rules): every stored block adds
  * lr * delta~_i x~_j^T; the inner checksums follow the same rule so they stay valid. */
+static void update_impl(orc_layer_t* L, const float* Delta, const float* X, int B, float lr, int small, uint32_t iteration);
 void orc_update(orc_layer_t* L, const float* Delta, const float* X, int B, float lr) {
+  update_impl(L, Delta, X, B, lr, 0, 0u);
+}
+
+static void update_impl(orc_layer_t* L, const float* Delta, const float* X, int B, float lr, int small, uint32_t iteration) {
   const int br = L->b_r, bc = L->b_c, M = L->M, Nn = L->Nn;
   float* Xt = (float*)malloc((size_t)B * Nn * bc * sizeof(float));
   float* Dt = (float*)malloc((size_t)B * M * br * sizeof(float));
   orc_encode_x(L, X, B, Xt);
   orc_encode_delta(L, Delta, B, Dt);
+  if (small && L->have_small) {
+    /* soft errors in the additional encoding: the whole encoded sub-vector of a hit parity index is off; the
+     * update (blocks and inner checksums alike) takes the erroneous vector, so the stored parity blocks of that
+     * block-column / block-row leave the code and the next products on them show it */
+    const orc_small_faults_t* sf = &L->small;
+    for (int j = L->d.n; j < Nn; ++j)
+      if (orc_small_hit(sf, ORC_PHASE_ENCODE, iteration, (uint32_t)j))
+        for (int c = 0; c < bc; ++c)
+          for (int b = 0; b < B; ++b)
+            Xt[(size_t)b * Nn * bc + j * bc + c] += orc_noise(sf->seed, sf->layer, ORC_PHASE_ENCODE, iteration, (uint32_t)j,
+                                                            (uint32_t)(c * B + b), sf->sigma);
+    for (int i = L->d.m; i < M; ++i)
+      if (orc_small_hit(sf, ORC_PHASE_ENCODE, iteration, (uint32_t)(Nn + i)))
+        for (int r = 0; r < br; ++r)
+          for (int b = 0; b < B; ++b)
+            Dt[(size_t)b * M * br + i * br + r] += orc_noise(sf->seed, sf->layer, ORC_PHASE_ENCODE, iteration, (uint32_t)(Nn + i),
+                                                           (uint32_t)(r * B + b), sf->sigma);
+  }
   const double eta = (double)lr;
 #pragma omp parallel for collapse(2) schedule(dynamic)
   for (int i = 0; i < M; ++i)
@@ -924,6 +1017,7 @@ void orc_backward_update(orc_layer_t* L, const float* Delta, const float* X, int
   float* Z = (float*)malloc(total * sizeof(float));
   float* Zc = (float*)malloc(total * sizeof(float));
   uint64_t inj[64];
+  L->small_iteration = iteration;
   orc_backward_products(L, Delta, B, Z); /* uses the weights of this iteration, before O3 */
   memcpy(Zc, Z, total * sizeof(float));
   orc_inject(L, ORC_PHASE_BWD, f, iteration, Z, B, inj);
@@ -939,7 +1033,7 @@ void orc_backward_update(orc_layer_t* L, const float* Delta, const float* X, int
         C[(size_t)b * L->d.n_in + g] = (float)acc;
       }
   free(Z); free(Zc);
-  orc_update(L, Delta, X, B, lr);
+  update_impl(L, Delta, X, B, lr, 1, iteration);
 }
 
 void orc_decode_weights(const orc_layer_t* L, float* W_out) {

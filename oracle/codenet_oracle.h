@@ -34,7 +34,9 @@ enum { ORC_LOCATE_NONE = 0, ORC_LOCATE_SYNDROME = 1, ORC_LOCATE_NODECHECK = 2,
        ORC_LOCATE_JOINT = 4 /* syndrome-only, supports of up to r - 1 nodes (vector errors); 3 is not used here */ };
 enum { ORC_FAULT_NONE = 0, ORC_FAULT_BERNOULLI = 1, ORC_FAULT_EXACTLY_ONE = 2 };
 enum { ORC_PHASE_FWD = 0, ORC_PHASE_BWD = 1 };
-enum { ORC_CLEAN = 0, ORC_CORRECTED = 1, ORC_FALLBACK = 2, ORC_FAILED = 3 };
+enum { ORC_CLEAN = 0, ORC_CORRECTED = 1, ORC_FALLBACK = 2, ORC_FAILED = 3,
+       ORC_DISAGREE = 5 /* a verification step found two evaluations that differ: restore the last checkpoint */ };
+enum { ORC_PHASE_ENCODE = 2, ORC_PHASE_INPUT = 3, ORC_PHASE_CHECK = 4, ORC_PHASE_DECODE = 5 };  /* small steps */
 enum { ORC_ACT_IDENTITY = 0, ORC_ACT_RELU = 1 };
 enum { ORC_LOSS_MSE_MEAN = 0, ORC_LOSS_SOFTMAX_CE = 1 };
 
@@ -55,6 +57,19 @@ typedef struct {
   uint32_t seed, layer, mode, p_q32;
   float sigma;
 } orc_fault_t;
+
+/* Soft errors in the steps around the products (Error Model 2 in the additional encoding, in the generation of a
+ * node's input sub-vector by the activation / post-multiplication step, in error detection and in decoding;
+ * Section "Decentralized Implementation").  Unit u of phase ph is hit in an iteration when word 0 of
+ * Philox(counter (iteration, u, 0, 0), key (seed, layer << 8 | ph)) is below the phase's p_q32; noise values come
+ * from orc_noise with the same key.  Units: ENCODE: j for x~_j (j >= n), Nn + i for delta~_i (i >= m), drawn in the
+ * backward call; INPUT: node i * Nn + j of the feedforward products (its own copy of x_j is off by a noise vector,
+ * so its output is off by W~_ij times that vector); CHECK and DECODE: the codeword, per phase of the call. */
+typedef struct {
+  uint32_t seed, layer;
+  uint32_t p_encode_q32, p_input_q32, p_check_q32, p_decode_q32;
+  float sigma;
+} orc_small_faults_t;
 
 typedef struct {
   uint32_t status;
@@ -123,6 +138,10 @@ void orc_backward_update(orc_layer_t* L, const float* Delta, const float* X, int
                          const orc_fault_t* f, uint32_t iteration, float* C, orc_report_t* rep);
 
 void orc_decode_weights(const orc_layer_t* L, float* W_out /* n_out x n_in */);
+/* Plan for soft errors in the small steps of every later call on this layer (copied; NULL: none). */
+void orc_layer_set_small_faults(orc_layer_t* L, const orc_small_faults_t* plan);
+/* Was unit `unit` of small-step phase `phase` hit in `iteration` under `plan`? */
+int orc_small_hit(const orc_small_faults_t* plan, uint32_t phase, uint32_t iteration, uint32_t unit);
 double orc_check_invariance(const orc_layer_t* L);
 /* Conditioning of the erasure decoding of the code of one direction (phase 0: G_r, phase 1: G_c), over every square
  * sub-system of the parity part with at most r unknowns: out[0] worst ||A||_inf ||A^-1||_inf, out[1] worst

@@ -48,6 +48,11 @@ class Fault(C.Structure):
                 ("p_q32", C.c_uint32), ("sigma", C.c_float)]
 
 
+class SmallFaults(C.Structure):
+    _fields_ = [("seed", C.c_uint32), ("layer", C.c_uint32), ("p_encode_q32", C.c_uint32), ("p_input_q32", C.c_uint32),
+                ("p_check_q32", C.c_uint32), ("p_decode_q32", C.c_uint32), ("sigma", C.c_float)]
+
+
 class Report(C.Structure):
     _fields_ = [("status", C.c_uint32), ("n_detected_cw", C.c_uint32),
                 ("n_flagged_nodes", C.c_uint32), ("n_fallback_cw", C.c_uint32),
@@ -107,6 +112,10 @@ def lib():
     L.orc_backward_update.argtypes = [vp, fp, fp, C.c_int, C.c_float, C.POINTER(Fault),
                                       C.c_uint32, fp, C.POINTER(Report)]
     L.orc_decode_weights.argtypes = [vp, fp]
+    L.orc_layer_set_small_faults.argtypes = [vp, C.POINTER(SmallFaults)]
+    L.orc_layer_set_small_faults.restype = None
+    L.orc_small_hit.argtypes = [C.POINTER(SmallFaults), C.c_uint32, C.c_uint32, C.c_uint32]
+    L.orc_small_hit.restype = C.c_int
     L.orc_code_conditioning.argtypes = [vp, C.c_int, C.POINTER(C.c_double)]
     L.orc_code_conditioning.restype = None
     L.orc_check_invariance.argtypes = [vp]
@@ -151,6 +160,19 @@ def noise(seed, layer, phase, iteration, node_id, element, sigma):
 def make_fault(seed=0, layer=0, mode=FAULT_NONE, p=0.0, sigma=10.0):
     p_q32 = min(int(p * 4294967296.0), 0xFFFFFFFF)
     return Fault(seed, layer, mode, p_q32, sigma)
+
+
+DISAGREE = 5
+PHASE_ENCODE, PHASE_INPUT, PHASE_CHECK, PHASE_DECODE = 2, 3, 4, 5
+
+
+def make_small_faults(seed=0, layer=0, p_encode=0.0, p_input=0.0, p_check=0.0, p_decode=0.0, sigma=10.0):
+    q = lambda p: min(int(p * 4294967296.0), 0xFFFFFFFF)
+    return SmallFaults(seed, layer, q(p_encode), q(p_input), q(p_check), q(p_decode), sigma)
+
+
+def small_hit(plan, phase, iteration, unit):
+    return bool(lib().orc_small_hit(C.byref(plan), phase, iteration, unit))
 
 
 def node_hit(fault, phase, iteration, node_id, active_index, n_active):
@@ -311,6 +333,11 @@ class Layer:
         W = np.empty((self.n_out, self.n_in), np.float32)
         lib().orc_decode_weights(self.h, _fp(W))
         return W
+
+    def set_small_faults(self, plan):
+        """Soft errors in the small steps (encoding, input copies, detection, decoding) of every later call; None: off."""
+        self._small = plan
+        lib().orc_layer_set_small_faults(self.h, None if plan is None else C.byref(plan))
 
     def code_conditioning(self, phase):
         """(worst condition number, worst ||A^-1||, worst error amplification) over the erasure sub-systems."""

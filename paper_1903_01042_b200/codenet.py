@@ -17,7 +17,8 @@ MATH_FFMA, MATH_TF32, MATH_BF16 = 0, 1, 2
 LOCATE_NONE, LOCATE_SYNDROME, LOCATE_NODECHECK, LOCATE_OFF, LOCATE_JOINT = 0, 1, 2, 3, 4
 FAULT_NONE, FAULT_BERNOULLI, FAULT_EXACTLY_ONE = 0, 1, 2
 PHASE_FWD, PHASE_BWD = 0, 1
-CLEAN, CORRECTED, FALLBACK, FAILED, TIMEOUT = 0, 1, 2, 3, 4
+CLEAN, CORRECTED, FALLBACK, FAILED, TIMEOUT, DISAGREE = 0, 1, 2, 3, 4, 5
+PHASE_ENCODE, PHASE_INPUT, PHASE_CHECK, PHASE_DECODE = 2, 3, 4, 5
 ACT_IDENTITY, ACT_RELU = 0, 1
 LOSS_MSE_MEAN, LOSS_SOFTMAX_CE = 0, 1
 MAX_NODES = 64
@@ -35,6 +36,12 @@ class LayerDesc(C.Structure):
 class Fault(C.Structure):
     _fields_ = [("seed", C.c_uint32), ("layer", C.c_uint32), ("mode", C.c_uint32),
                 ("p_q32", C.c_uint32), ("sigma", C.c_float), ("iteration_dev", C.c_void_p)]
+
+
+class SmallFaults(C.Structure):
+    _fields_ = [("seed", C.c_uint32), ("layer", C.c_uint32), ("p_encode_q32", C.c_uint32), ("p_input_q32", C.c_uint32),
+                ("p_check_q32", C.c_uint32), ("p_decode_q32", C.c_uint32), ("sigma", C.c_float),
+                ("iteration_dev", C.c_void_p)]
 
 
 class Report(C.Structure):
@@ -100,6 +107,8 @@ def lib():
     L.codenet_layer_dims.argtypes = [vp, C.POINTER(C.c_int32)]
     L.codenet_code_conditioning.argtypes = [vp, ip, C.POINTER(C.c_double)]
     L.codenet_code_conditioning.restype = ip
+    L.codenet_layer_set_small_faults.argtypes = [vp, C.POINTER(SmallFaults)]
+    L.codenet_layer_set_small_faults.restype = ip
     L.codenet_set_wait_limit.argtypes = [C.c_uint64, vp]
     L.codenet_set_wait_limit.restype = ip
     L.codenet_withhold_tile_loads.argtypes = [ip, vp]
@@ -374,6 +383,20 @@ def withhold_tile_loads(on):
 
 def reset_timeout(layer):
     _check(lib().codenet_reset_timeout(layer.h, _stream()))
+
+
+def make_small_faults(seed=0, layer=0, p_encode=0.0, p_input=0.0, p_check=0.0, p_decode=0.0, sigma=10.0,
+                      iteration_dev=None):
+    """Plan for soft errors in the small steps; ``iteration_dev`` as in make_fault."""
+    q = lambda p: min(int(p * 4294967296.0), 0xFFFFFFFF)
+    return SmallFaults(seed, layer, q(p_encode), q(p_input), q(p_check), q(p_decode), sigma,
+                       None if iteration_dev is None else iteration_dev.data_ptr())
+
+
+def set_small_faults(layer, plan):
+    """codenet_layer_set_small_faults: applies to every later call on the layer; None switches it off."""
+    layer._small = plan
+    _check(lib().codenet_layer_set_small_faults(layer.h, None if plan is None else C.byref(plan)))
 
 
 def check_invariance(layer):

@@ -38,6 +38,8 @@ struct CheckParams {
   int out_act;             // forward sums: activation applied as they are written (step C1), or identity
   const float* out_mask;   // backward sums: zeroed where this input is not positive (step C2), or NULL
   uint32_t* bump;          // iteration counter of the fault plans to advance when the kernel ends, or NULL
+  SmallDev small;          // soft errors in the small steps (input copies, the two verification steps); on == 0: none
+  const float* dY;         // output deviations of the nodes whose input copy is hit [codeword][node][len][B], or NULL
 };
 
 struct PhaseGeom {
@@ -159,24 +161,48 @@ __device__ __forceinline__ uint32_t node_id_of(const Geom& g, int phase, int cw,
   return (uint32_t)(i * g.Nn + j);
 }
 
-// Which nodes of every codeword the injection plan hits, into shared memory.
-__device__ void build_hit_masks(const CheckParams& p, const PhaseGeom& q, unsigned long long* s_inj) {
-  for (int t = threadIdx.x; t < MAXN; t += blockDim.x) s_inj[t] = 0ull;
+// Which nodes of every codeword are erroneous, into shared memory: s_inj = the nodes whose output the injection
+// plan hits or (feedforward) whose own input copy the small-step plan hits; s_out / s_in (may be NULL) tell the two
+// kinds apart for the code that builds the working copy.
+__device__ void build_hit_masks(const CheckParams& p, const PhaseGeom& q, unsigned long long* s_inj,
+                                unsigned long long* s_out = nullptr, unsigned long long* s_in = nullptr) {
+  for (int t = threadIdx.x; t < MAXN; t += blockDim.x) {
+    s_inj[t] = 0ull;
+    if (s_out) s_out[t] = 0ull;
+    if (s_in) s_in[t] = 0ull;
+  }
   __syncthreads();
-  if (p.fault.mode != CODENET_FAULT_NONE) {
+  const bool fwd = p.phase == CODENET_PHASE_FWD;
+  const bool inputs = fwd && p.small.on && p.small.p_input != 0u && p.dY != nullptr;
+  if (p.fault.mode != CODENET_FAULT_NONE || inputs) {
     const uint32_t it = p.fault.iteration ? *p.fault.iteration : 0u;
-    const bool fwd = p.phase == CODENET_PHASE_FWD;
+    const uint32_t its = p.small.iteration ? *p.small.iteration : 0u;
     const uint32_t n_active = (uint32_t)(q.n_cw * q.K);
     for (int t = threadIdx.x; t < q.n_cw * q.K; t += blockDim.x) {
       const int cw = t / q.K, k = t % q.K;
       const int i = fwd ? k : cw, j = fwd ? cw : k;
       const uint32_t node_id = (uint32_t)(i * p.g.Nn + j);
       const uint32_t active = fwd ? (uint32_t)(i * p.g.n + j) : node_id;
-      if (node_is_hit(p.fault, (uint32_t)p.phase, it, node_id, active, n_active))
+      if (p.fault.mode != CODENET_FAULT_NONE && node_is_hit(p.fault, (uint32_t)p.phase, it, node_id, active, n_active)) {
         atomicOr(&s_inj[cw], 1ull << k);
+        if (s_out) atomicOr(&s_out[cw], 1ull << k);
+      }
+      if (inputs && small_is_hit(p.small, CODENET_PHASE_INPUT, its, node_id)) {
+        atomicOr(&s_inj[cw], 1ull << k);
+        if (s_in) atomicOr(&s_in[cw], 1ull << k);
+      }
     }
   }
   __syncthreads();
+}
+
+// The value of element e of a node output as the checks see it: the product, plus the noise of an erroneous output,
+// plus the deviation an erroneous input copy causes (in that order, each one rounding).
+__device__ __forceinline__ float with_faults(const CheckParams& p, float v, bool out_hit, bool in_hit, uint32_t key1,
+                                             uint32_t it, uint32_t node_id, size_t node_base, size_t e) {
+  if (out_hit) v = __fadd_rn(v, hit_noise(p.fault.seed, key1, it, node_id, (uint32_t)e, p.fault.sigma));
+  if (in_hit) v = __fadd_rn(v, p.dY[node_base + e]);
+  return v;
 }
 
 __device__ __forceinline__ float block_max256(float v, float* red) {
@@ -313,6 +339,7 @@ __device__ void write_report(const CheckParams& p, int n_cw, const unsigned* fin
       uint32_t outcome = CODENET_CLEAN;
       if (state == 1) outcome = CODENET_CORRECTED;
       else if (state == 3) outcome = p.have_clean ? CODENET_FALLBACK : CODENET_FAILED;
+      else if (state == 4) outcome = CODENET_DISAGREE;
       const unsigned long long F = pl.F;
       rep->flagged_mask[cw] = pl.detected ? F : 0ull;
       rep->injected_mask[cw] = pl.injected;
@@ -361,7 +388,7 @@ __device__ __forceinline__ float final_value(const CheckParams& p, const PhaseGe
                                              int node, size_t e) {
   const CwView yw = cw_view(p, q, s_inj, cw);
   const int state = (int)s_final[cw];
-  if (state == 0) return yw.at(q, node, e);
+  if (state == 0 || state == 4) return yw.at(q, node, e);   // (4: the verification steps disagreed: left as it is)
   if (state == 1) {
     const CwPlan& pl = p.plan[cw];
     if (!((pl.F >> node) & 1ull)) return yw.at(q, node, e);

@@ -36,6 +36,7 @@ void free_layer_memory(codenet_layer* L) {
   cudaFree(L->ws.Xt); cudaFree(L->ws.Dt); cudaFree(L->ws.dsum); cudaFree(L->ws.xsum);
   cudaFree(L->ws.tc_x); cudaFree(L->ws.tc_d); cudaFree(L->ws.tc_dT); cudaFree(L->ws.tc_xT); cudaFree(L->ws.tc_flag); cudaFree(L->ws.chk);
   cudaFree(L->ws.Y); cudaFree(L->ws.Yw); cudaFree(L->ws.Ynext); cudaFree(L->ws.stats); cudaFree(L->ws.plan);
+  cudaFree(L->ws.dY);
 }
 
 int cuda_status(cudaError_t e) {
@@ -228,6 +229,7 @@ int codenet_encode_layer(const codenet_layer_desc_t* d, const void* W_dev, coden
   L->next_x = nullptr;
   L->next_B = 0;
   L->ws.Ynext = nullptr;
+  L->ws.dY = nullptr;
   L->ws.tc_x = nullptr;
   L->ws.tc_d = nullptr;
   L->ws.tc_dT = nullptr;
@@ -355,6 +357,7 @@ int codenet_forward(codenet_layer_t* L, const float* X_dev, int B, const codenet
   const bool have_next = L->next_x != nullptr && L->next_x == X_dev && L->next_B == B;
   L->next_x = nullptr;
   if (have_next) {
+    CN_TRY(launch_input_faults(*L, B, st));
     CN_TRY(launch_check(*L, CODENET_PHASE_FWD, L->ws.Ynext, 2, L->ws.Yw, X_dev, B, inject ? &fd : nullptr, 1, 0,
                         S_dev, 0.0f, 0, rep_dev, st));
     return CODENET_OK;
@@ -366,7 +369,9 @@ int codenet_forward(codenet_layer_t* L, const float* X_dev, int B, const codenet
   }
   if (tc_forward_supported(g, L->desc.math, B)) CN_TRY(launch_tc_forward(*L, X_dev, B, L->ws.Y, st));
   else CN_TRY(launch_forward_products(g, x, ldx, B, L->ws.Y, st));
-  const bool checks = inject || (g.locate_mode != CODENET_LOCATE_OFF && (g.r_row > 0 || g.locate_mode == CODENET_LOCATE_NODECHECK));
+  const bool checks = inject || L->small.on ||
+                      (g.locate_mode != CODENET_LOCATE_OFF && (g.r_row > 0 || g.locate_mode == CODENET_LOCATE_NODECHECK));
+  if (checks) CN_TRY(launch_input_faults(*L, B, st));
   if (checks)
     CN_TRY(launch_check(*L, CODENET_PHASE_FWD, L->ws.Y, 0, L->ws.Yw, X_dev, B, inject ? &fd : nullptr, 1, 0, S_dev,
                         0.0f, 0, rep_dev, st));
@@ -406,7 +411,7 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
   const Geom& g = L->g;
   // the operand copies of the fused tensor-core kernel ride on the vector encoding
   const int emit = (B > 8 && tc_backward_update_supported(g, L->desc.math, B)) ? (g.dtype == CODENET_F32 ? 1 : 2) : 0;
-  CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit));
+  CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit, L->small.on ? &L->small : nullptr));
   int src_kind;
   if (B <= 8) {
     const bool next = X_next_dev != nullptr && L->next_ok &&
@@ -460,6 +465,26 @@ int codenet_regenerate_block(codenet_layer_t* L, int i, int j, int along, codene
   }
   CN_TRY(launch_regenerate_block(g, i, j, along, nullptr, reinterpret_cast<cudaStream_t>(stream)));
   L->next_x = nullptr;
+  return CODENET_OK;
+}
+
+int codenet_layer_set_small_faults(codenet_layer_t* L, const codenet_small_faults_t* plan) {
+  if (!L) return CODENET_E_BADARG;
+  if (plan == nullptr) { L->small.on = 0; return CODENET_OK; }
+  if (plan->p_input_q32 != 0u && L->ws.dY == nullptr) {
+    // the deviations of the nodes with an erroneous input copy need a buffer of the size of the node outputs
+    const size_t elems = (size_t)L->g.n * L->g.Mbr * (size_t)L->batch_max;
+    if (cudaMalloc(reinterpret_cast<void**>(&L->ws.dY), elems * sizeof(float)) != cudaSuccess) {
+      cudaGetLastError();
+      L->ws.dY = nullptr;
+      return CODENET_E_NOMEM;
+    }
+  }
+  L->small.seed = plan->seed; L->small.layer = plan->layer;
+  L->small.p_encode = plan->p_encode_q32; L->small.p_input = plan->p_input_q32;
+  L->small.p_check = plan->p_check_q32; L->small.p_decode = plan->p_decode_q32;
+  L->small.sigma = plan->sigma; L->small.iteration = plan->iteration_dev;
+  L->small.on = 1;
   return CODENET_OK;
 }
 

@@ -42,6 +42,14 @@ struct FaultDev {
   const uint32_t* iteration;
 };
 
+// Soft errors in the small steps (codenet_small_faults_t on the device side); on == 0: none.
+struct SmallDev {
+  uint32_t seed, layer, p_encode, p_input, p_check, p_decode;
+  float sigma;
+  const uint32_t* iteration;
+  int on;
+};
+
 // Statistics gathered across CTAs by the check kernel (floats as ordered unsigned bit patterns,
 // combined with atomicMax so the result does not depend on arrival order).
 struct CheckStats {
@@ -79,6 +87,7 @@ struct Workspace {
   int* tc_flag;   // [0] set by a tensor-core kernel whose bounded wait ran out; [1] which statistics buffer the
                   // next check kernel works in (kept on the device, flipped by the kernel)
   float* chk;     // inner-check scratch for batches > 8 (check_scratch_floats), or NULL
+  float* dY;      // output deviations W~_ij nu of nodes whose input copy is hit, [codeword][node][len][B], or NULL
   CheckStats* stats;  // two buffers used alternately; each check clears the other one
   CwPlan* plan;       // one per codeword
   size_t y_elems, yw_elems;
@@ -103,6 +112,7 @@ struct codenet_layer {
   mutable const float* out_mask;
   // a recorded step's iteration counter: the backward check of the step's last layer advances it itself when
   // no other kernel of the step reads it afterwards (bump_done tells the recorder that it did)
+  codenet::SmallDev small = {0, 0, 0, 0, 0, 0, 0.0f, nullptr, 0};   // soft errors in the small steps
   mutable int operands_ready = 0;   // the vector-encoding kernel has written the tensor-core operand copies
   mutable uint32_t* bump_after = nullptr;
   mutable bool bump_done = false;
@@ -168,8 +178,12 @@ struct LossFuse {
 // emit: 0 = the fp32 vectors only; 1 = also their transposes (rows, B) for the fused TF32 kernel; 2 = also the
 // bfloat16 copies the fused bf16 kernel reads (delta~ as a hi / lo pair, x~ rounded).  Sets L.operands_ready
 // when the extra copies were written (the 16-byte path only).
+// small != NULL: soft errors in the additional encoding (the parity sub-vectors of hit units get noise)
 cudaError_t launch_encode_vectors(const codenet_layer_impl& L, const float* X, const float* Delta,
-                                  int B, cudaStream_t st, const LossFuse* fuse = nullptr, int emit = 0);
+                                  int B, cudaStream_t st, const LossFuse* fuse = nullptr, int emit = 0,
+                                  const SmallDev* small = nullptr);
+// Output deviations of the feedforward nodes whose own input copy the plan hits, into L.ws.dY (zeroed first).
+cudaError_t launch_input_faults(const codenet_layer_impl& L, int B, cudaStream_t st);
 // Injection, detection, location, decoding plan and the final sums over codewords.
 // src_kind: 0 = canonical [cw][node][len][B] in `src`; 1 = backward partials [i][rt][b][ld];
 // 2 = feedforward partials [strip][coded row][b] with ldb / strip-width strips per block-column.
@@ -241,6 +255,15 @@ __device__ __forceinline__ bool node_is_hit(const FaultDev& f, uint32_t phase, u
   }
   philox4x32_10(iteration, 0xFFFFFFFFu, 0u, 0u, f.seed, key1, o);
   return (o[0] % n_active) == active_index;
+}
+
+__device__ __forceinline__ bool small_is_hit(const SmallDev& sf, uint32_t phase, uint32_t iteration, uint32_t unit) {
+  const uint32_t pq = phase == CODENET_PHASE_ENCODE ? sf.p_encode : phase == CODENET_PHASE_INPUT ? sf.p_input
+                    : phase == CODENET_PHASE_CHECK ? sf.p_check : sf.p_decode;
+  if (!sf.on || pq == 0u) return false;
+  uint32_t o[4];
+  philox4x32_10(iteration, unit, 0u, 0u, sf.seed, (sf.layer << 8) | phase, o);
+  return o[0] < pq;
 }
 
 __device__ __forceinline__ float warp_sum(float v) {

@@ -46,11 +46,16 @@ __global__ void encode_layer_kernel(Geom g, const void* __restrict__ W) {
 }
 
 // Inner checksums of the stored blocks: u = column sums per slice of T rows, v = row sums.
-__global__ void checksum_kernel(Geom g) {
+// only_blk >= 0: the checksums of that block alone (regeneration), otherwise of every block (initial encoding).
+__global__ void checksum_kernel(Geom g, int only_blk) {
   const size_t nu = (size_t)g.M * g.Nn * g.ns * g.ldb;
   const size_t nv = (size_t)g.M * g.Nn * g.nsc * g.b_r;
-  for (size_t idx = blockIdx.x * (size_t)blockDim.x + threadIdx.x; idx < nu + nv;
-       idx += (size_t)gridDim.x * blockDim.x) {
+  const size_t per_u = (size_t)g.ns * g.ldb, per_v = (size_t)g.nsc * g.b_r;
+  const size_t count = only_blk >= 0 ? per_u + per_v : nu + nv;
+  for (size_t it = blockIdx.x * (size_t)blockDim.x + threadIdx.x; it < count; it += (size_t)gridDim.x * blockDim.x) {
+    // position in the full index space (all u entries, then all v entries)
+    const size_t idx = only_blk < 0 ? it
+                       : (it < per_u ? (size_t)only_blk * per_u + it : nu + (size_t)only_blk * per_v + (it - per_u));
     if (idx < nu) {
       const int c = (int)(idx % g.ldb);
       const size_t t = idx / g.ldb;
@@ -93,9 +98,9 @@ struct EmitOperands {
 __global__ void __launch_bounds__(128)
 encode_vectors_kernel(Geom g, const float* __restrict__ X, const float* __restrict__ Delta, int B,
                       float* __restrict__ Xt, float* __restrict__ Dt, float* __restrict__ dsum,
-                      float* __restrict__ xsum, int vec_ok, LossFuse lf, EmitOperands em) {
+                      float* __restrict__ xsum, int vec_ok, LossFuse lf, EmitOperands em, SmallDev sf) {
   __shared__ float red[4];
-  __shared__ int s_last;
+  __shared__ int s_last, s_enc_hit;
   const int nxseg = X ? g.Nn * g.nsc * B : 0;
   int seg = blockIdx.x;
   float part = 0.0f, loss_part = 0.0f;
@@ -137,6 +142,14 @@ encode_vectors_kernel(Geom g, const float* __restrict__ X, const float* __restri
       if (i < g.m) loss_id = (i * g.ns + sl) * B + b;
     }
   }
+  // soft error in the additional encoding: the whole parity sub-vector of a hit unit is off by noise
+  const int seg_b = (blockIdx.x < nxseg ? blockIdx.x : blockIdx.x - nxseg) % B;
+  const uint32_t enc_unit = blockIdx.x < nxseg ? (uint32_t)k : (uint32_t)(g.Nn + k);
+  const uint32_t enc_it = sf.iteration ? *sf.iteration : 0u;
+  if (threadIdx.x == 0) s_enc_hit = (k >= kd && small_is_hit(sf, CODENET_PHASE_ENCODE, enc_it, enc_unit)) ? 1 : 0;
+  __syncthreads();
+  const bool enc_hit = s_enc_hit != 0;
+  const uint32_t enc_key = (sf.layer << 8) | (uint32_t)CODENET_PHASE_ENCODE;
   const float scale = lf.scale;
   if (vec_ok) {
     // four entries per thread and step: lengths, offsets and pointers are multiples of four floats
@@ -165,6 +178,12 @@ encode_vectors_kernel(Geom g, const float* __restrict__ X, const float* __restri
             v.x = fmaf(c, t.x, v.x); v.y = fmaf(c, t.y, v.y); v.z = fmaf(c, t.z, v.z); v.w = fmaf(c, t.w, v.w);
           }
         }
+      }
+      if (enc_hit && e < len) {
+        v.x = __fadd_rn(v.x, soft_error_noise(sf.seed, enc_key, enc_it, enc_unit, (uint32_t)(e * B + seg_b), sf.sigma));
+        v.y = __fadd_rn(v.y, soft_error_noise(sf.seed, enc_key, enc_it, enc_unit, (uint32_t)((e + 1) * B + seg_b), sf.sigma));
+        v.z = __fadd_rn(v.z, soft_error_noise(sf.seed, enc_key, enc_it, enc_unit, (uint32_t)((e + 2) * B + seg_b), sf.sigma));
+        v.w = __fadd_rn(v.w, soft_error_noise(sf.seed, enc_key, enc_it, enc_unit, (uint32_t)((e + 3) * B + seg_b), sf.sigma));
       }
       *reinterpret_cast<float4*>(dst + e) = v;
       if (tr) {
@@ -207,6 +226,7 @@ encode_vectors_kernel(Geom g, const float* __restrict__ X, const float* __restri
           }
         }
       }
+      if (enc_hit && e < len) v = __fadd_rn(v, soft_error_noise(sf.seed, enc_key, enc_it, enc_unit, (uint32_t)(e * B + seg_b), sf.sigma));
       dst[e] = v;
       part += v;
     }
@@ -514,13 +534,13 @@ inline int grid_for(size_t n, int threads) {
 cudaError_t launch_encode_layer(const Geom& g, const void* W, cudaStream_t st) {
   encode_layer_kernel<<<grid_for((size_t)g.Mbr * g.ld, 256), 256, 0, st>>>(g, W);
   const size_t nchk = (size_t)g.M * g.Nn * ((size_t)g.ns * g.ldb + (size_t)g.nsc * g.b_r);
-  checksum_kernel<<<grid_for(nchk, 128), 128, 0, st>>>(g);
+  checksum_kernel<<<grid_for(nchk, 128), 128, 0, st>>>(g, -1);
   count_launch(2);
   return cudaGetLastError();
 }
 
 cudaError_t launch_encode_vectors(const codenet_layer_impl& L, const float* X, const float* Delta,
-                                  int B, cudaStream_t st, const LossFuse* fuse, int emit) {
+                                  int B, cudaStream_t st, const LossFuse* fuse, int emit, const SmallDev* small) {
   const Geom& g = L.g;
   const int nseg = (X ? g.Nn * g.nsc * B : 0) + (Delta ? g.M * g.ns * B : 0);
   if (nseg == 0) return cudaSuccess;
@@ -541,7 +561,9 @@ cudaError_t launch_encode_vectors(const codenet_layer_impl& L, const float* X, c
     else { em.xb = reinterpret_cast<__nv_bfloat16*>(L.ws.tc_xT); em.dpair = reinterpret_cast<__nv_bfloat16*>(L.ws.tc_d); }
     L.operands_ready = (em.xT || em.xb) ? 1 : 0;
   }
-  encode_vectors_kernel<<<nseg, 128, 0, st>>>(g, X, Delta, B, L.ws.Xt, L.ws.Dt, L.ws.dsum, L.ws.xsum, vec_ok ? 1 : 0, lf, em);
+  SmallDev sf = {0, 0, 0, 0, 0, 0, 0.0f, nullptr, 0};
+  if (small != nullptr) sf = *small;
+  encode_vectors_kernel<<<nseg, 128, 0, st>>>(g, X, Delta, B, L.ws.Xt, L.ws.Dt, L.ws.dsum, L.ws.xsum, vec_ok ? 1 : 0, lf, em, sf);
   count_launch();
   return cudaGetLastError();
 }
@@ -595,7 +617,9 @@ cudaError_t launch_regenerate_block(const Geom& g, int i, int j, int along, int*
   ProfileScope scope(CODENET_KERNEL_REGENERATE, st);
   if (g.dtype == CODENET_BF16) regenerate_block_kernel<__nv_bfloat16><<<(int)blocks, 256, 0, st>>>(g, i, j, along, status_dev);
   else regenerate_block_kernel<float><<<(int)blocks, 256, 0, st>>>(g, i, j, along, status_dev);
-  count_launch();
+  // everything the node stored is generated again: its inner checksums follow from the rebuilt block
+  checksum_kernel<<<grid_for((size_t)g.ns * g.ldb + (size_t)g.nsc * g.b_r, 128), 128, 0, st>>>(g, i * g.Nn + j);
+  count_launch(2);
   return cudaGetLastError();
 }
 

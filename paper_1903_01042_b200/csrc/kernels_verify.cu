@@ -58,7 +58,8 @@ __device__ __forceinline__ float warp_sum32(float (&v2)[4][8]) {
 // BIG_SR rows of it and 32 batch entries: node norm and the slice sums of the inner check.  Only nodes the
 // injection plan hits get noise and a working copy; the others stay where the product kernel wrote them.
 __device__ __forceinline__ void big_phase_u(const CheckParams& p, const PhaseGeom& q,
-                                            const unsigned long long* s_inj, uint32_t it, uint32_t key1,
+                                            const unsigned long long* s_inj, const unsigned long long* s_out,
+                                            const unsigned long long* s_in, uint32_t it, uint32_t key1,
                                             bool node_check, int nrch, int NS) {
   const Geom& g = p.g;
   const int B = p.B, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -77,7 +78,7 @@ __device__ __forceinline__ void big_phase_u(const CheckParams& p, const PhaseGeo
     const int rc = rest % nrch, s = rest / nrch;
     const int b = gq * 32 + lb;
     const int t_begin = rc * BIG_SR, t_end = min(t_begin + BIG_SR, q.slen);
-    const bool hit = (s_inj[cw] >> k) & 1ull;
+    const bool hit = (s_inj[cw] >> k) & 1ull, h_out = (s_out[cw] >> k) & 1ull, h_in = (s_in[cw] >> k) & 1ull;
     const size_t nb = ((size_t)cw * q.K + k) * q.n_el;
     const float* src = p.src + nb;
     float* yw = p.Yw + nb;
@@ -96,10 +97,10 @@ __device__ __forceinline__ void big_phase_u(const CheckParams& p, const PhaseGeo
           const int t = t0 + w * rpl + lr;
           if (t >= t_end) continue;
           const size_t e = ((size_t)s * q.slen + t) * B + b;
-          v[w].x = __fadd_rn(v[w].x, hit_noise(p.fault.seed, key1, it, node_id, (uint32_t)e, p.fault.sigma));
-          v[w].y = __fadd_rn(v[w].y, hit_noise(p.fault.seed, key1, it, node_id, (uint32_t)(e + 1), p.fault.sigma));
-          v[w].z = __fadd_rn(v[w].z, hit_noise(p.fault.seed, key1, it, node_id, (uint32_t)(e + 2), p.fault.sigma));
-          v[w].w = __fadd_rn(v[w].w, hit_noise(p.fault.seed, key1, it, node_id, (uint32_t)(e + 3), p.fault.sigma));
+          v[w].x = with_faults(p, v[w].x, h_out, h_in, key1, it, node_id, nb, e);
+          v[w].y = with_faults(p, v[w].y, h_out, h_in, key1, it, node_id, nb, e + 1);
+          v[w].z = with_faults(p, v[w].z, h_out, h_in, key1, it, node_id, nb, e + 2);
+          v[w].w = with_faults(p, v[w].w, h_out, h_in, key1, it, node_id, nb, e + 3);
           *reinterpret_cast<float4*>(yw + e) = v[w];
         }
       }
@@ -353,11 +354,11 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
   constexpr bool big_batch = BIG;  // the host launches this instantiation exactly when lazy_copy(p) holds
 
   __shared__ float sP[MAXN * MAXR];
-  __shared__ unsigned long long s_inj[MAXN];
+  __shared__ unsigned long long s_inj[MAXN], s_out[MAXN], s_in[MAXN];
   __shared__ unsigned s_syn[MAXN];
   __shared__ float red[CK_WARPS];
   __shared__ float s_proj[MAXR * MAXR];
-  __shared__ int s_state, s_cand_ok, s_accept;
+  __shared__ int s_state, s_cand_ok, s_accept, s_verify;
   __shared__ unsigned long long s_F;
   __shared__ float s_tau, s_scale, s_smax, s_h;
   __shared__ float s_nrm[MAXN], s_rat[MAXN];
@@ -365,7 +366,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
 
   for (int t = tid; t < q.kd * q.r; t += CK_THREADS) sP[t] = q.P[t];
   for (int t = tid; t < MAXN; t += CK_THREADS) s_syn[t] = 0u;
-  build_hit_masks(p, q, s_inj);
+  build_hit_masks(p, q, s_inj, s_out, s_in);
   if (tid == 0) {
     // h = max_t (1 + sum_k |P[k, t]|), the code's part of the syndrome threshold (read in phase D)
     float h = 0.0f;
@@ -392,16 +393,17 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     const int ncch = (dlen + BIG_DC - 1) / BIG_DC;                          // chunks of it
     const int NS = 2 * nrch + 2 * ncch;                                     // scratch floats per (unit, b)
     if (by_bgroup) {
-      big_phase_u(p, q, s_inj, it, key1, node_check, nrch, NS);
+      big_phase_u(p, q, s_inj, s_out, s_in, it, key1, node_check, nrch, NS);
     }
     // units go round the CTAs first and then round the warps, so that a few hundred of them spread over
     // all SMs instead of filling the first CTAs
     for (int unit = blockIdx.x + gridDim.x * warp; unit < (by_bgroup ? 0 : n_units); unit += gridDim.x * CK_WARPS) {
       const int s = unit % q.nsl, ck = unit / q.nsl;
       const int k = ck % q.K, cw = ck / q.K;
-      const bool hit = (s_inj[cw] >> k) & 1ull;
+      const bool hit = (s_inj[cw] >> k) & 1ull, h_out = (s_out[cw] >> k) & 1ull, h_in = (s_in[cw] >> k) & 1ull;
       const uint32_t node_id = node_id_of(g, p.phase, cw, k);
-      float* yw = p.Yw + ((size_t)cw * q.K + k) * q.n_el;
+      const size_t nb = ((size_t)cw * q.K + k) * q.n_el;
+      float* yw = p.Yw + nb;
       const size_t e0 = (size_t)s * SL;
       const bool copy = !(p.src_kind == 0 && p.src == p.Yw && !hit);
       float mx = 0.0f;
@@ -456,7 +458,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
             if (t >= SL) continue;
             const size_t e = e0 + t;
             if (copy) {
-              if (hit) v[u] = __fadd_rn(v[u], hit_noise(p.fault.seed, key1, it, node_id, (uint32_t)e, p.fault.sigma));
+              if (hit) v[u] = with_faults(p, v[u], h_out, h_in, key1, it, node_id, nb, e);
               yw[e] = v[u];
             }
             mx = fmaxf(mx, fabsf(v[u]));
@@ -477,7 +479,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
         float v;
         if (copy) {
           v = clean_value(p, q, cw, k, e);
-          if (hit) v = __fadd_rn(v, hit_noise(p.fault.seed, key1, it, node_id, (uint32_t)e, p.fault.sigma));
+          if (hit) v = with_faults(p, v, h_out, h_in, key1, it, node_id, nb, e);
           yw[e] = v;
         } else {
           v = yw[e];
@@ -999,10 +1001,23 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       else if (flags != 0) s_state = 1;
       else if (g.locate_mode != CODENET_LOCATE_NONE && q.r >= 2) s_state = 2;
       else s_state = 3;
+      // Verification step of the error detection ("Errors in Error-Detection under Error Model 2"): the evaluation
+      // of the codeword's parity checks is made twice and compared.  A soft error in one evaluation shifts its
+      // value by a noise sample; any difference means the evaluations disagree: the codeword is left as it is and
+      // the caller restores the last checkpoint.
+      s_verify = 0;
+      if (p.small.on) {
+        const uint32_t its = p.small.iteration ? *p.small.iteration : 0u;
+        const uint32_t vunit = (uint32_t)(p.phase * 64 + cw);
+        if (small_is_hit(p.small, CODENET_PHASE_CHECK, its, vunit) &&
+            hit_noise(p.small.seed, (p.small.layer << 8) | (uint32_t)CODENET_PHASE_CHECK, its, vunit, 0u, p.small.sigma) != 0.0f)
+          s_verify = 1;
+      }
       }
     __syncthreads();
-    int state = s_state;  // block-uniform copy
-    const bool detected = state != 0;
+    const bool disagree_check = s_verify != 0;
+    int state = disagree_check ? 4 : s_state;  // block-uniform copy
+    const bool detected = state != 0 && !disagree_check;
 
     // location from the syndrome alone: smallest support (<= r/2 nodes, lexicographic order) whose
     // least-squares fit leaves a residual below tau
@@ -1095,6 +1110,19 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       pl.max_clean = cw_max_clean;
       pl.nfd = 0;
       pl.spare = 0;
+      if (detected && p.small.on) {
+        // Verification step of the decoding ("Errors in decoding under Error Model 2"): the list of nodes found
+        // erroneous is made twice and compared.  A soft error in one evaluation changes the membership of one node
+        // (chosen by the generator): the lists differ and the decoding is deemed erroneous.
+        const uint32_t its = p.small.iteration ? *p.small.iteration : 0u;
+        const uint32_t vunit = (uint32_t)(p.phase * 64 + cw);
+        if (small_is_hit(p.small, CODENET_PHASE_DECODE, its, vunit)) {
+          uint32_t o[4];
+          philox4x32_10(its, vunit, 1u, 0u, p.small.seed, (p.small.layer << 8) | (uint32_t)CODENET_PHASE_DECODE, o);
+          const unsigned long long F_other = F ^ (1ull << (o[0] % (uint32_t)q.K));
+          if (F_other != F) state = 4;
+        }
+      }
       if (state == 1) {
         int nfd = 0, nq = 0, ok = 1;
         if (__popcll(F) > q.r) ok = 0;
@@ -1134,6 +1162,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
         if (state == 3) atomicAdd(&r->n_fallback_cw, 1u);
         const uint32_t outcome = state == 1 ? (uint32_t)CODENET_CORRECTED
                                : state == 3 ? (uint32_t)(p.have_clean ? CODENET_FALLBACK : CODENET_FAILED)
+                               : state == 4 ? (uint32_t)CODENET_DISAGREE
                                             : (uint32_t)CODENET_CLEAN;
         if (outcome != CODENET_CLEAN) atomicMax(&r->status, outcome);
         atomicMin(reinterpret_cast<unsigned*>(&r->min_margin_hit), __float_as_uint(cw_min_hit));
@@ -1313,6 +1342,32 @@ __global__ void __launch_bounds__(CK_THREADS) fix_kernel(CheckParams p) {
   }
 }
 
+// Soft errors in a node's own copy of its input sub-vector (the copy the activation / post-multiplication step
+// generated for it): the node multiplies W~_ij (x_j + nu), so its output is off by W~_ij nu.  One CTA per
+// (feedforward node, slab of 32 columns): a hit node's slab of nu goes to shared memory, every row's partial product
+// is added into dY (zeroed before the launch; the order of the additions is not fixed: the node is located and its
+// output discarded, only the size of the deviation matters).
+__global__ void __launch_bounds__(256) input_fault_kernel(Geom g, SmallDev sf, int B, float* __restrict__ dY) {
+  extern __shared__ float s_nu[];   // [32 columns][B]
+  const int node = blockIdx.x, j = node / g.M, i = node % g.M;   // codeword (block-column) j, node (block-row) i
+  const uint32_t its = sf.iteration ? *sf.iteration : 0u;
+  const uint32_t node_id = (uint32_t)(i * g.Nn + j);
+  if (!small_is_hit(sf, CODENET_PHASE_INPUT, its, node_id)) return;
+  const int c0 = blockIdx.y * 32, nc = min(32, g.b_c - c0);
+  const uint32_t key1 = (sf.layer << 8) | (uint32_t)CODENET_PHASE_INPUT;
+  for (int t = threadIdx.x; t < nc * B; t += blockDim.x)
+    s_nu[t] = soft_error_noise(sf.seed, key1, its, node_id, (uint32_t)((c0 + t / B) * B + t % B), sf.sigma);
+  __syncthreads();
+  float* out = dY + ((size_t)j * g.M + i) * ((size_t)g.b_r * B);
+  for (int t = threadIdx.x; t < g.b_r * B; t += blockDim.x) {
+    const int r = t / B, b = t % B;
+    float acc = 0.0f;
+    for (int c = 0; c < nc; ++c)
+      acc = fmaf(load_elem(g.Wt, g.dtype, ((size_t)i * g.b_r + r) * g.ld + (size_t)j * g.ldb + c0 + c), s_nu[c * B + b], acc);
+    atomicAdd(out + t, acc);
+  }
+}
+
 // Plain sums of the data-node outputs for calls that check nothing (no code, or the checks switched off, and no
 // injection): s_i = sum_j y_ij / c_j = sum_i z_ij straight from the node outputs or their partial sums, in the same
 // fixed order as the checked path, an empty report.  No barrier, no working copy, no inner-checksum update.
@@ -1396,6 +1451,7 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
   p.Xt = L.ws.Xt; p.Dt = L.ws.Dt; p.dsum = L.ws.dsum; p.xsum = L.ws.xsum;
   p.st = nullptr; p.st_next = nullptr; p.st_base = L.ws.stats; p.parity = L.ws.tc_flag + 1;
   p.plan = L.ws.plan; p.rep = rep; p.tc_flag = L.ws.tc_flag; p.chk = L.ws.chk;
+  p.small = L.small; p.dY = L.ws.dY;
   p.out_act = phase == CODENET_PHASE_FWD ? L.out_act : CODENET_ACT_IDENTITY;
   p.out_mask = phase == CODENET_PHASE_BWD ? L.out_mask : nullptr;
   if (phase == CODENET_PHASE_FWD) L.out_act = CODENET_ACT_IDENTITY; else L.out_mask = nullptr;
@@ -1404,7 +1460,7 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
   const bool fwd = phase == CODENET_PHASE_FWD;
   const bool phase_unchecked = g.locate_mode == CODENET_LOCATE_OFF ||
                                ((fwd ? g.r_row : g.r_col) == 0 && g.locate_mode != CODENET_LOCATE_NODECHECK);
-  if (fault == nullptr && out != nullptr && have_clean && !commit && phase_unchecked &&
+  if (fault == nullptr && !L.small.on && out != nullptr && have_clean && !commit && phase_unchecked &&
       (!update_checksums || !keeps_checksums(g))) {
     // nothing to inject and nothing to decide: the sums alone, one plain launch (the inner checksums are left
     // alone where nothing can read them: keeps_checksums)
@@ -1465,6 +1521,17 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
   }
   count_launch();
   return e;
+}
+
+cudaError_t launch_input_faults(const codenet_layer_impl& L, int B, cudaStream_t st) {
+  const Geom& g = L.g;
+  if (!L.small.on || L.small.p_input == 0u || L.ws.dY == nullptr) return cudaSuccess;
+  cudaError_t e = cudaMemsetAsync(L.ws.dY, 0, (size_t)g.n * g.Mbr * B * sizeof(float), st);
+  if (e != cudaSuccess) return e;
+  dim3 grid(g.n * g.M, (g.b_c + 31) / 32);
+  input_fault_kernel<<<grid, 256, (size_t)32 * B * sizeof(float), st>>>(g, L.small, B, L.ws.dY);
+  count_launch();
+  return cudaGetLastError();
 }
 
 cudaError_t launch_sum_outputs(const Geom& g, int phase, int B, const float* Y, float* out, int out_act,

@@ -346,6 +346,100 @@ def test_a_bounded_wait_that_runs_out_is_reported_and_the_layer_recovers(cn, orc
     assert _rel(S.cpu().numpy(), So) <= TOL_LOWP
 
 
+@pytest.mark.parametrize("shape,B,bf16,math", [((96, 60, 3, 4, 2, 2, True), 2, False, 0),
+                                                ((192, 256, 2, 2, 1, 1, False), 1, False, 0),
+                                                ((512, 512, 2, 2, 2, 2, True), 64, False, 1)])
+def test_soft_errors_in_the_small_steps_against_the_oracle(cn, orc, shape, B, bf16, math):
+    """Error Model 2 in the steps around the products (additional encoding, a node's own input copy, error
+    detection, decoding) with the two verification steps: the same generator drives both sides, so the reports must
+    agree step by step (DISAGREE included), outputs must agree whenever the call was not told to roll back, and
+    the stored blocks, which encoding errors push out of the code, must stay equal on both sides.  After a
+    DISAGREE both sides restore their checkpoint, as the method prescribes."""
+    no, ni, m, n, rr, rc, gauss = shape
+    W = wl.weights(no, ni, seed=71, bf16=bf16)
+    Pr, Pc = _codes(m, n, rr, rc, gauss)
+    p = Pair(cn, orc, W, m, n, rr, rc, Pr, Pc, bf16=bf16, batch_max=B, math=math)
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kw = dict(seed=8, layer=2, p_encode=0.04, p_input=0.03, p_check=0.04, p_decode=0.3, sigma=10.0)
+    cn.set_small_faults(p.g, cn.make_small_faults(iteration_dev=it_dev, **kw))
+    p.o.set_small_faults(orc.make_small_faults(**kw))
+    fg = cn.make_fault(seed=12, layer=2, mode=cn.FAULT_BERNOULLI, p=0.04, sigma=10.0, iteration_dev=it_dev)
+    fo = orc.make_fault(seed=12, layer=2, mode=orc.FAULT_BERNOULLI, p=0.04, sigma=10.0)
+    rep = cn.new_reports(1)
+    repb = cn.new_reports(1)
+    tol = TOL_LOWP if math else TOL_F32
+    seen = {"disagree": 0, "input": 0, "encode": 0}
+    cn.checkpoint_save(p.g)
+    p.o.checkpoint_save()
+    for it in range(60):
+        X = wl.gaussian_inputs(B, ni, seed=72, iteration=it)
+        D = wl.gaussian_inputs(B, no, seed=73, iteration=it) / np.float32(B)
+        it_dev.fill_(it)
+        S = cn.forward(p.g, _dev(X), fault=fg, rep_dev=rep)
+        Cg = cn.backward_update(p.g, _dev(D), _dev(X), 0.02, fault=fg, rep_dev=repb)
+        So, ro = p.o.forward(X, fo, it)
+        Co, rbo = p.o.backward_update(D, X, 0.02, fo, it)
+        rf, rb = cn.read_reports(rep)[0], cn.read_reports(repb)[0]
+        assert rf.decisions() == ro.decisions(), ("forward", it, rf.decisions()[:5], ro.decisions()[:5])
+        assert rb.decisions() == rbo.decisions(), ("backward", it, rb.decisions()[:5], rbo.decisions()[:5])
+        loose = TOL_DECODED if gauss else tol
+        if rf.status != cn.DISAGREE:
+            assert _rel(S.cpu().numpy(), So) <= (max(tol, loose) if rf.status != cn.CLEAN else tol), it
+        if rb.status != cn.DISAGREE:
+            assert _rel(Cg.cpu().numpy(), Co) <= (max(tol, loose) if rb.status != cn.CLEAN else tol), it
+        Nn = n + rc
+        seen["input"] += any(orc.small_hit(p.o._small, orc.PHASE_INPUT, it, i * Nn + j) for i in range(m + rr) for j in range(n))
+        seen["encode"] += any(orc.small_hit(p.o._small, orc.PHASE_ENCODE, it, u) for u in list(range(n, Nn)) + [Nn + i for i in range(m, m + rr)])
+        if rf.status == cn.DISAGREE or rb.status == cn.DISAGREE:
+            seen["disagree"] += 1
+            cn.checkpoint_restore(p.g)
+            p.o.checkpoint_restore()
+        elif it % 10 == 9:
+            cn.checkpoint_save(p.g)
+            p.o.checkpoint_save()
+        if it % 10 == 0:
+            # stored blocks (pushed out of the code by encoding errors, identically on both sides) and checksums
+            for (i, j) in [(0, 0), (m, 0), (0, n), (m + rr - 1, n - 1), (m - 1, n + rc - 1)]:
+                got = cn.get_block(p.g, i, j).cpu().numpy()
+                assert _rel(got, p.o.block(i, j)) <= (1e-4 if not math else 5e-3), (it, i, j)
+    assert min(seen.values()) > 0, seen
+
+
+def test_regeneration_rebuilds_the_inner_checksums_of_the_block(cn, orc):
+    """Everything a regenerated node stored is generated again: after an encoding error has entered a parity block
+    and its inner checksums through the update, regeneration restores both, as on the oracle (up to the one
+    rounding by which the two sides' updated data blocks may differ)."""
+    m, n, r = 2, 3, 2
+    W = wl.weights(64, 96, seed=81)
+    Pr, Pc = _codes(m, n, r, r, True)
+    p = Pair(cn, orc, W, m, n, r, r, Pr, Pc, batch_max=2)
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kw = dict(seed=3, layer=0, p_encode=1.0, sigma=10.0)          # every parity sub-vector is hit once
+    X = wl.gaussian_inputs(2, 96, seed=82)
+    D = wl.gaussian_inputs(2, 64, seed=83)
+    cn.set_small_faults(p.g, cn.make_small_faults(iteration_dev=it_dev, **kw))
+    p.o.set_small_faults(orc.make_small_faults(**kw))
+    cn.backward_update(p.g, _dev(D), _dev(X), 0.05)
+    p.o.backward_update(D, X, 0.05)
+    cn.set_small_faults(p.g, None)
+    p.o.set_small_faults(None)
+    assert cn.check_invariance(p.g) > 1e-2 and p.o.check_invariance() > 1e-2
+    for j in range(n):
+        for i in range(m, m + r):
+            cn.regenerate_block(p.g, i, j, 0)
+            p.o.regenerate_block(i, j, 0)
+    for i in range(m):
+        for j in range(n, n + r):
+            cn.regenerate_block(p.g, i, j, 1)
+            p.o.regenerate_block(i, j, 1)
+    assert cn.check_invariance(p.g) < 1e-5 and p.o.check_invariance() < 1e-5
+    p.compare_checksums(cn, 1e-6)
+    for i in range(m + r):
+        for j in range(n + r):
+            if p.o.has_node(i, j):
+                assert _rel(cn.get_block(p.g, i, j).cpu().numpy(), p.o.block(i, j)) <= 1e-6, (i, j)
+
+
 def test_check_rows_slices(cn, orc):
     W = wl.weights(64, 32, seed=12)
     p = Pair(cn, orc, W, 2, 2, 1, 1, batch_max=2, check_rows=8, check_cols=4)

@@ -638,6 +638,136 @@ def test_node_check_threshold_has_a_rounding_floor_for_cancelling_checksums(orc)
 
 
 # ---------------------------------------------------------------------------------------------
+# soft errors in the small steps (Error Model 2 in encoding, input generation, detection, decoding)
+# ---------------------------------------------------------------------------------------------
+
+def _small_layer(orc, m=2, n=2, r=2, b=6, seed=3, mode=None):
+    from paper_1903_01042_b200 import workloads as wl
+    rng = np.random.default_rng(seed)
+    W = rng.standard_normal((m * b, n * b)).astype(np.float32)
+    Pr, Pc = wl.gaussian_parity(m, r, seed, 0), wl.gaussian_parity(n, r, seed, 1)
+    lay = orc.Layer(W, m, n, r, r, P_row=Pr, P_col=Pc, locate_mode=orc.LOCATE_NODECHECK if mode is None else mode, tau_rel=1e-3)
+    return lay, W, rng
+
+
+def _iteration_hitting_only(orc, plan, phase, units, wanted, start=0):
+    """First iteration >= start in which exactly the units in `wanted` (of all `units`) are hit."""
+    for it in range(start, start + 100000):
+        if {u for u in units if orc.small_hit(plan, phase, it, u)} == set(wanted):
+            return it
+    raise AssertionError("no such iteration")
+
+
+def test_encoding_faults_surface_at_the_next_products_and_are_repaired(orc):
+    """A soft error in the additional encoding (delta~_i of a parity block-row, x~_j of a parity block-column) does
+    not touch the products of its own iteration; it enters the stored parity blocks through the update, and the
+    next products that use those blocks show it in every codeword, at exactly that parity node (Section
+    "Decentralized Implementation", last paragraph).  Every single encoding unit of the 2 x 2 + 2 + 2 grid is tried
+    in turn.  Regeneration of the affected blocks (or the checkpoint) brings the layer back into the code."""
+    m = n = 2
+    for unit in range(4):                      # x~_2, x~_3 (units 2, 3), delta~_2, delta~_3 (units Nn + 2, Nn + 3)
+        lay, W, rng = _small_layer(orc, mode=orc.LOCATE_SYNDROME)
+        Nn = n + 2
+        units = [n, n + 1, Nn + m, Nn + m + 1]
+        plan = orc.make_small_faults(seed=5, layer=1, p_encode=0.3, sigma=10.0)
+        it = _iteration_hitting_only(orc, plan, orc.PHASE_ENCODE, units, [units[unit]])
+        X = rng.standard_normal((2, n * 6)).astype(np.float32)
+        D = rng.standard_normal((2, m * 6)).astype(np.float32)
+        lay.checkpoint_save()
+        lay.set_small_faults(plan)
+        S, rf = lay.forward(X, None, it)
+        C, rb = lay.backward_update(D, X, 0.05, None, it)
+        lay.set_small_faults(None)
+        assert rf.status == orc.CLEAN and rb.status == orc.CLEAN       # nothing shows in the iteration of the fault
+        assert lay.check_invariance() > 1e-2                            # but the stored parity blocks left the code
+        S2, rf2 = lay.forward(X, None, it + 1)
+        C2, rb2 = lay.backward_update(D, X, 0.0, None, it + 1)
+        if unit < 2:      # x~_j entered the blocks of parity block-column j: the backward products show it
+            j = units[unit]
+            assert rf2.status == orc.CLEAN
+            assert rb2.n_detected_cw == m and all(rb2.flagged_mask[i] == 1 << j for i in range(m))
+            assert rb2.status == orc.CORRECTED
+            for i in range(m):
+                lay.regenerate_block(i, j, 1)
+        else:             # delta~_i entered the blocks of parity block-row i: the feedforward products show it
+            i = units[unit] - Nn
+            assert rf2.n_detected_cw == n and all(rf2.flagged_mask[j] == 1 << i for j in range(n))
+            assert rf2.status == orc.CORRECTED and rb2.status == orc.CLEAN
+            for j in range(n):
+                lay.regenerate_block(i, j, 0)
+        # corrected outputs are the plain products with the (intact) data blocks
+        assert _rel(S2, X.astype(np.float64) @ lay.decode_weights().astype(np.float64).T) < 1e-4
+        assert lay.check_invariance() < 1e-5
+        S3, rf3 = lay.forward(X, None, it + 2)
+        C3, rb3 = lay.backward_update(D, X, 0.0, None, it + 2)
+        assert rf3.status == orc.CLEAN and rb3.status == orc.CLEAN
+        lay.checkpoint_restore()                                        # the other remedy: back to the checkpoint
+        assert lay.check_invariance() < 1e-6 and _rel(lay.decode_weights(), W) == 0.0
+
+
+def test_input_copy_faults_are_located_like_output_faults(orc):
+    """A node whose own copy of its input sub-vector is off (an error in the activation / post-multiplication step
+    that generated it) outputs W~_ij (x_j + nu): the deviation W~_ij nu is caught by the same checks as any
+    erroneous output, in the same call.  Every single node of the 2 x 2 + 2 + 2 grid in turn, then a random run."""
+    lay, W, rng = _small_layer(orc)
+    m = n = 2
+    M, Nn = 4, 4
+    nodes = [i * Nn + j for i in range(M) for j in range(n)]
+    plan = orc.make_small_faults(seed=9, layer=0, p_input=0.1, sigma=10.0)
+    lay.set_small_faults(plan)
+    X = rng.standard_normal((3, n * 6)).astype(np.float32)
+    want = X.astype(np.float64) @ W.astype(np.float64).T
+    for node in nodes:
+        it = _iteration_hitting_only(orc, plan, orc.PHASE_INPUT, nodes, [node])
+        S, rep = lay.forward(X, None, it)
+        i, j = node // Nn, node % Nn
+        assert rep.status == orc.CORRECTED and rep.n_detected_cw == 1
+        assert rep.injected_mask[j] == 1 << i and rep.flagged_mask[j] == 1 << i
+        assert rep.min_margin_hit > 10.0 and _rel(S, want) < 1e-4
+    hits = 0
+    for it in range(200):
+        S, rep = lay.forward(X, None, it)
+        truth = [sum(1 << i for i in range(M) if orc.small_hit(plan, orc.PHASE_INPUT, it, i * Nn + j)) for j in range(n)]
+        assert list(rep.injected_mask[:n]) == truth
+        hits += sum(bin(t).count("1") for t in truth)
+        if all(bin(t).count("1") <= 2 for t in truth):
+            assert list(rep.flagged_mask[:n]) == truth and _rel(S, want) < 1e-4
+    assert hits > 50
+
+
+def test_verification_steps_report_a_disagreement_exactly_when_an_evaluation_was_hit(orc):
+    """The two verification steps: a soft error in one evaluation of a codeword's parity checks, or (for a
+    detected codeword) of its list of erroneous nodes, makes the evaluations differ; the call then reports
+    DISAGREE (the caller restores the last checkpoint).  Ground truth is the generator; without a plan, or with
+    nothing hit, the status never appears."""
+    lay, W, rng = _small_layer(orc)
+    m = n = 2
+    X = rng.standard_normal((2, n * 6)).astype(np.float32)
+    D = rng.standard_normal((2, m * 6)).astype(np.float32)
+    f = orc.make_fault(seed=4, mode=orc.FAULT_BERNOULLI, p=0.15, sigma=10.0)
+    plan = orc.make_small_faults(seed=6, layer=0, p_check=0.1, p_decode=0.3, sigma=10.0)
+    seen = {"check": 0, "decode": 0, "none": 0}
+    for it in range(300):
+        lay.set_small_faults(None)
+        S0, r0 = lay.forward(X, f, it)                                   # the same call without small-step errors
+        assert r0.status != orc.DISAGREE
+        lay.set_small_faults(plan)
+        S, rep = lay.forward(X, f, it)
+        hit_c = [orc.small_hit(plan, orc.PHASE_CHECK, it, 0 * 64 + cw) for cw in range(n)]
+        hit_d = [orc.small_hit(plan, orc.PHASE_DECODE, it, 0 * 64 + cw) and bool((r0.detected_mask >> cw) & 1) and not hit_c[cw]
+                 for cw in range(n)]
+        assert (rep.status == orc.DISAGREE) == (any(hit_c) or any(hit_d)), it
+        seen["check"] += any(hit_c); seen["decode"] += any(hit_d); seen["none"] += not (any(hit_c) or any(hit_d))
+        if not (any(hit_c) or any(hit_d)):
+            assert rep.decisions() == r0.decisions() and np.array_equal(S, S0)
+        C, rb = lay.backward_update(D, X, 0.0, f, it)
+        hit_cb = [orc.small_hit(plan, orc.PHASE_CHECK, it, 1 * 64 + cw) for cw in range(m)]
+        if any(hit_cb):
+            assert rb.status == orc.DISAGREE
+    assert min(seen.values()) > 10
+
+
+# ---------------------------------------------------------------------------------------------
 # bfloat16 storage
 # ---------------------------------------------------------------------------------------------
 
