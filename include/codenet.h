@@ -193,6 +193,22 @@ int codenet_backward_update_next(codenet_layer_t* layer, const float* Delta_dev,
                                  codenet_report_t* rep_dev, const float* X_next_dev,
                                  codenet_stream_t stream);
 
+/* As codenet_backward_update_next followed by codenet_forward(layer, X_next_dev, B, fault_next, S_next_dev,
+ * rep_next_dev): the backpropagation product, checks and update of this iteration (Algorithm 1,
+ * backpropagation loop and update stage) and the whole feedforward stage of the next one (Algorithm 1,
+ * feedforward loop) on the blocks just updated.  The two checks decide on independent codewords (block-rows of
+ * this iteration's products, block-columns of the next one's), so for batch 1 with the node check and at most
+ * one parity per code they share one launch; otherwise the two calls are made one after the other: the results
+ * are the same either way.  The forward stage belongs to the NEXT iteration: its fault plan's device counter is
+ * read plus one (the counter is advanced only after this call), so fault_next may point at the same plan as
+ * `fault`.  S_next_dev: (B, n_out) receives W_new x_next; rep_next_dev (may be NULL) its report.
+ * Errors: BADARG (also X_next_dev or S_next_dev NULL). */
+int codenet_backward_update_forward_next(codenet_layer_t* layer, const float* Delta_dev, const float* X_dev,
+                                         int B, float lr, const codenet_fault_t* fault, float* C_dev,
+                                         codenet_report_t* rep_dev, const float* X_next_dev,
+                                         const codenet_fault_t* fault_next, float* S_next_dev,
+                                         codenet_report_t* rep_next_dev, codenet_stream_t stream);
+
 /* Fault in the stored weights, as in the paper's own experiment (Section "Experimental Results": a
  * sparse matrix is added to the sub-matrix a node stores).  Element e = row * (N_in/n) + col of coded
  * block (i, j) changes when word 0 of Philox4x32-10(counter = (iteration, i * (n + r_col) + j, e, 3),
@@ -261,7 +277,9 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
                  codenet_stream_t stream);
 
 /* Announce the input of the NEXT codenet_step (device pointer, (B, n_in of layer 1)); the coming step
- * then uses codenet_backward_update_next on layer 1.  One-shot: cleared by that step. */
+ * then uses codenet_backward_update_next on layer 1 (codenet_backward_update_forward_next where that
+ * call shares a launch: the next step, given the announced pointer, then finds layer 1's forward stage done;
+ * its sums and report appear where this interface says when that step ends).  One-shot: cleared by that step. */
 int codenet_net_set_next_input(codenet_net_t* net, const float* X_next_dev);
 
 /* Record one codenet_step (same arguments; X_next_dev as in codenet_net_set_next_input, or NULL) into a

@@ -87,6 +87,8 @@ def lib():
     L.codenet_forward.argtypes = [vp, vp, ip, C.POINTER(Fault), vp, vp, vp]
     L.codenet_backward_update.argtypes = [vp, vp, vp, ip, fl, C.POINTER(Fault), vp, vp, vp]
     L.codenet_backward_update_next.argtypes = [vp, vp, vp, ip, fl, C.POINTER(Fault), vp, vp, vp, vp]
+    L.codenet_backward_update_forward_next.argtypes = [vp, vp, vp, ip, fl, C.POINTER(Fault), vp, vp, vp,
+                                                       C.POINTER(Fault), vp, vp, vp]
     L.codenet_net_set_next_input.argtypes = [vp, vp]
     L.codenet_net_capture_step.argtypes = [vp, vp, vp, ip, fl, C.POINTER(Fault), vp, vp, vp, vp, C.POINTER(ip)]
     L.codenet_net_replay.argtypes = [vp, ip, vp]
@@ -123,7 +125,7 @@ def lib():
                  "codenet_detect_decode", "codenet_net_create", "codenet_step",
                  "codenet_decode_weights", "codenet_check_invariance", "codenet_get_block",
                  "codenet_layer_dims", "codenet_net_output", "codenet_get_checksums",
-                 "codenet_backward_update_next", "codenet_net_set_next_input", "codenet_net_capture_step",
+                 "codenet_backward_update_next", "codenet_backward_update_forward_next", "codenet_net_set_next_input", "codenet_net_capture_step",
                  "codenet_net_replay", "codenet_corrupt_block", "codenet_regenerate_block",
                  "codenet_checkpoint_save", "codenet_checkpoint_restore"):
         getattr(L, name).restype = ip
@@ -275,6 +277,27 @@ def backward_update(layer, Delta_dev, X_dev, lr, fault=None, C_dev=None, rep_dev
                                                   None if fault is None else C.byref(fault), _ptr(C_dev),
                                                   _ptr(rep_dev), _ptr(X_next_dev), _stream()))
     return C_dev
+
+
+def backward_update_forward_next(layer, Delta_dev, X_dev, lr, X_next_dev, fault=None, fault_next=None, C_dev=None,
+                                 rep_dev=None, S_next_dev=None, rep_next_dev=None):
+    """codenet_backward_update_forward_next: this iteration's backward product, checks and update and the next
+    iteration's whole forward stage; returns (C_dev, S_next_dev)."""
+    B = X_dev.shape[0]
+    _dev_f32(X_dev, (B, layer.n_in))
+    _dev_f32(X_next_dev, (B, layer.n_in))
+    _dev_f32(Delta_dev, (B, layer.n_out))
+    if C_dev is None:
+        C_dev = torch.empty((B, layer.n_in), dtype=torch.float32, device=X_dev.device)
+    if S_next_dev is None:
+        S_next_dev = torch.empty((B, layer.n_out), dtype=torch.float32, device=X_dev.device)
+    _dev_f32(C_dev, (B, layer.n_in))
+    _dev_f32(S_next_dev, (B, layer.n_out))
+    _check(lib().codenet_backward_update_forward_next(
+        layer.h, _ptr(Delta_dev), _ptr(X_dev), B, float(lr), None if fault is None else C.byref(fault), _ptr(C_dev),
+        _ptr(rep_dev), _ptr(X_next_dev), None if fault_next is None else C.byref(fault_next), _ptr(S_next_dev),
+        _ptr(rep_next_dev), _stream()))
+    return C_dev, S_next_dev
 
 
 def detect_decode(layer, phase, Y_dev, V_dev, rep_dev=None):

@@ -40,6 +40,13 @@ struct CheckParams {
   uint32_t* bump;          // iteration counter of the fault plans to advance when the kernel ends, or NULL
   SmallDev small;          // soft errors in the small steps (input copies, the two verification steps); on == 0: none
   const float* dY;         // output deviations of the nodes whose input copy is hit [codeword][node][len][B], or NULL
+  // --- paired launch (the backward check of one iteration and the forward check of the next in one kernel) ---
+  uint32_t it_add;         // added to the fault plan's counter: 1 for the look-ahead forward check, whose
+                           // iteration starts only when the counter has been advanced
+  int pair;                // 0: a check of its own; 1: the backward part of a pair; 2: the forward part
+  float* pair_sums;        // forward part: [unit][2] slice sum and magnitude sum, from phase U to phase X
+  const float* commit_S; float* commit_S_to; int commit_n;   // forward part, on entry: sums and report of the
+  const codenet_report_t* commit_rep; codenet_report_t* commit_rep_to;   // previous pair go where the caller reads them
 };
 
 struct PhaseGeom {
@@ -175,7 +182,7 @@ __device__ void build_hit_masks(const CheckParams& p, const PhaseGeom& q, unsign
   const bool fwd = p.phase == CODENET_PHASE_FWD;
   const bool inputs = fwd && p.small.on && p.small.p_input != 0u && p.dY != nullptr;
   if (p.fault.mode != CODENET_FAULT_NONE || inputs) {
-    const uint32_t it = p.fault.iteration ? *p.fault.iteration : 0u;
+    const uint32_t it = (p.fault.iteration ? *p.fault.iteration : 0u) + p.it_add;
     const uint32_t its = p.small.iteration ? *p.small.iteration : 0u;
     const uint32_t n_active = (uint32_t)(q.n_cw * q.K);
     for (int t = threadIdx.x; t < q.n_cw * q.K; t += blockDim.x) {

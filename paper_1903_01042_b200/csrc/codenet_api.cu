@@ -14,6 +14,8 @@ struct codenet_net {
   std::vector<float*> xs;  // xs[l] = input of layer l for l >= 1 (library-owned)
   float* out_last;         // (B, n_L)
   const float* x_next;     // input of the next step, for layer 1's look-ahead products (one-shot)
+  float* s_stage;          // one-layer networks: sums of the next step's forward stage, done ahead by a paired check
+  codenet_report_t* rep_stage;   // its report, until the step it belongs to ends
   float* delta[2];         // ping-pong error vectors, (B, widest layer)
   float* loss_partials;    // 512 partial sums + one counter word (loss kernel), then LOSS_FUSE_PARTIALS + a counter (loss folded into the vector encoding)
   std::vector<cudaGraphExec_t> graphs;  // captured steps (codenet_net_capture_step)
@@ -35,7 +37,7 @@ void free_layer_memory(codenet_layer* L) {
   cudaFree(const_cast<float*>(L->g.Pr)); cudaFree(const_cast<float*>(L->g.Pc));
   cudaFree(L->ws.Xt); cudaFree(L->ws.Dt); cudaFree(L->ws.dsum); cudaFree(L->ws.xsum);
   cudaFree(L->ws.tc_x); cudaFree(L->ws.tc_d); cudaFree(L->ws.tc_dT); cudaFree(L->ws.tc_xT); cudaFree(L->ws.tc_flag); cudaFree(L->ws.chk);
-  cudaFree(L->ws.Y); cudaFree(L->ws.Yw); cudaFree(L->ws.Ynext); cudaFree(L->ws.stats); cudaFree(L->ws.plan);
+  cudaFree(L->ws.Y); cudaFree(L->ws.Yw); cudaFree(L->ws.Yw2); cudaFree(L->ws.pair_sums); cudaFree(L->ws.Ynext); cudaFree(L->ws.stats); cudaFree(L->ws.plan);
   cudaFree(L->ws.dY);
 }
 
@@ -301,9 +303,13 @@ int codenet_encode_layer(const codenet_layer_desc_t* d, const void* W_dev, coden
     if (L->next_ok) {
       const size_t strips = (size_t)g.n * g.ldb / backward_strip_elems(g.dtype);
       if ((e = dev_alloc(&ws.Ynext, strips * g.Mbr * Bs)) != cudaSuccess) break;
+      // a second working copy and the hand-over scratch for the forward part of a paired check (batch 1)
+      if ((e = dev_alloc(&ws.Yw2, (size_t)g.n * g.Mbr)) != cudaSuccess) break;
+      if ((e = dev_alloc(&ws.pair_sums, (size_t)2 * g.n * g.M * g.ns)) != cudaSuccess) break;
+      L->pair_ok = 1;
     }
-    if ((e = dev_alloc(&ws.stats, (size_t)2)) != cudaSuccess) break;
-    if ((e = dev_alloc(&ws.plan, (size_t)CODENET_MAX_NODES)) != cudaSuccess) break;
+    if ((e = dev_alloc(&ws.stats, (size_t)4)) != cudaSuccess) break;
+    if ((e = dev_alloc(&ws.plan, (size_t)2 * CODENET_MAX_NODES)) != cudaSuccess) break;
     std::vector<float> pr((size_t)g.m * (g.r_row > 0 ? g.r_row : 1), 1.0f);
     std::vector<float> pc((size_t)g.n * (g.r_col > 0 ? g.r_col : 1), 1.0f);
     if (d->P_row) for (int k = 0; k < g.m * g.r_row; ++k) pr[k] = d->P_row[k];
@@ -313,8 +319,8 @@ int codenet_encode_layer(const codenet_layer_desc_t* d, const void* W_dev, coden
     if ((e = cudaMemcpy(Pr, pr.data(), pr.size() * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
     if ((e = cudaMemcpy(Pc, pc.data(), pc.size() * sizeof(float), cudaMemcpyHostToDevice)) != cudaSuccess) break;
     if ((e = cudaMemsetAsync(g.Wt, 0, w_bytes, st)) != cudaSuccess) break;
-    if ((e = cudaMemsetAsync(ws.stats, 0, sizeof(CheckStats) * 2, st)) != cudaSuccess) break;
-    if ((e = cudaMemsetAsync(ws.plan, 0, sizeof(CwPlan) * CODENET_MAX_NODES, st)) != cudaSuccess) break;
+    if ((e = cudaMemsetAsync(ws.stats, 0, sizeof(CheckStats) * 4, st)) != cudaSuccess) break;
+    if ((e = cudaMemsetAsync(ws.plan, 0, sizeof(CwPlan) * 2 * CODENET_MAX_NODES, st)) != cudaSuccess) break;
     if ((e = launch_encode_layer(g, W_dev, st)) != cudaSuccess) break;
   } while (0);
   if (e != cudaSuccess) {
@@ -341,9 +347,19 @@ int codenet_layer_dims(const codenet_layer_t* L, int32_t dims[10]) {
   return CODENET_OK;
 }
 
+// it_add: added to the fault plan's device counter (1 when the call stands for the next iteration's forward stage)
+static int forward_impl(codenet_layer_t* L, const float* X_dev, int B, const codenet_fault_t* fault,
+                        float* S_dev, codenet_report_t* rep_dev, codenet_stream_t stream, uint32_t it_add);
+
 int codenet_forward(codenet_layer_t* L, const float* X_dev, int B, const codenet_fault_t* fault,
                     float* S_dev, codenet_report_t* rep_dev, codenet_stream_t stream) {
+  return forward_impl(L, X_dev, B, fault, S_dev, rep_dev, stream, 0u);
+}
+
+static int forward_impl(codenet_layer_t* L, const float* X_dev, int B, const codenet_fault_t* fault,
+                        float* S_dev, codenet_report_t* rep_dev, codenet_stream_t stream, uint32_t it_add) {
   if (!L || !X_dev || !S_dev || B < 1 || B > L->batch_max) return CODENET_E_BADARG;
+  L->pair_x = nullptr;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const Geom& g = L->g;
   // x can be read in place when no padding separates its sub-vectors
@@ -359,7 +375,7 @@ int codenet_forward(codenet_layer_t* L, const float* X_dev, int B, const codenet
   if (have_next) {
     CN_TRY(launch_input_faults(*L, B, st));
     CN_TRY(launch_check(*L, CODENET_PHASE_FWD, L->ws.Ynext, 2, L->ws.Yw, X_dev, B, inject ? &fd : nullptr, 1, 0,
-                        S_dev, 0.0f, 0, rep_dev, st));
+                        S_dev, 0.0f, 0, rep_dev, st, it_add));
     return CODENET_OK;
   }
   if (!direct) {
@@ -374,7 +390,7 @@ int codenet_forward(codenet_layer_t* L, const float* X_dev, int B, const codenet
   if (checks) CN_TRY(launch_input_faults(*L, B, st));
   if (checks)
     CN_TRY(launch_check(*L, CODENET_PHASE_FWD, L->ws.Y, 0, L->ws.Yw, X_dev, B, inject ? &fd : nullptr, 1, 0, S_dev,
-                        0.0f, 0, rep_dev, st));
+                        0.0f, 0, rep_dev, st, it_add));
   else {
     const int act = L->out_act;
     L->out_act = CODENET_ACT_IDENTITY;
@@ -391,10 +407,24 @@ int codenet_backward_update(codenet_layer_t* L, const float* Delta_dev, const fl
 
 // fuse != NULL: delta^L is formed from the last layer's sums and the target while the vectors are encoded
 // (Delta_dev receives it), see LossFuse.
+// pair != NULL: the forward stage of the next iteration (input X_next_dev) is wanted as well; where the layer allows
+// it (pair_supported, products taken ahead by the sweep) its check shares a launch with the backward check and
+// *paired is set, otherwise the caller runs it.
+struct PairWish {
+  const codenet_fault_t* fault_next;
+  float* S_next;
+  codenet_report_t* rep_next;
+  const float* commit_S; float* commit_S_to; int commit_n;
+  const codenet_report_t* commit_rep; codenet_report_t* commit_rep_to;
+};
 static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, const float* X_dev, int B,
                                 float lr, const codenet_fault_t* fault, float* C_dev,
                                 codenet_report_t* rep_dev, const float* X_next_dev, codenet_stream_t stream,
-                                const LossFuse* fuse);
+                                const LossFuse* fuse, const PairWish* pair = nullptr, bool* paired = nullptr);
+static bool lookahead_ok(const codenet_layer_t* L, const float* X_next_dev, int B) {
+  return X_next_dev != nullptr && B <= 8 && L->next_ok && (reinterpret_cast<uintptr_t>(X_next_dev) & 15u) == 0 &&
+         (L->g.n_in % 4) == 0;
+}
 
 int codenet_backward_update_next(codenet_layer_t* L, const float* Delta_dev, const float* X_dev, int B,
                                  float lr, const codenet_fault_t* fault, float* C_dev,
@@ -402,11 +432,29 @@ int codenet_backward_update_next(codenet_layer_t* L, const float* Delta_dev, con
   return backward_update_impl(L, Delta_dev, X_dev, B, lr, fault, C_dev, rep_dev, X_next_dev, stream, nullptr);
 }
 
+int codenet_backward_update_forward_next(codenet_layer_t* L, const float* Delta_dev, const float* X_dev, int B,
+                                         float lr, const codenet_fault_t* fault, float* C_dev,
+                                         codenet_report_t* rep_dev, const float* X_next_dev,
+                                         const codenet_fault_t* fault_next, float* S_next_dev,
+                                         codenet_report_t* rep_next_dev, codenet_stream_t stream) {
+  if (!X_next_dev || !S_next_dev) return CODENET_E_BADARG;
+  PairWish w;
+  memset(&w, 0, sizeof(w));
+  w.fault_next = fault_next; w.S_next = S_next_dev; w.rep_next = rep_next_dev;
+  bool paired = false;
+  const int rc = backward_update_impl(L, Delta_dev, X_dev, B, lr, fault, C_dev, rep_dev, X_next_dev, stream, nullptr,
+                                      &w, &paired);
+  if (rc != CODENET_OK || paired) return rc;
+  return forward_impl(L, X_next_dev, B, fault_next, S_next_dev, rep_next_dev, stream, 1u);
+}
+
 static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, const float* X_dev, int B,
                                 float lr, const codenet_fault_t* fault, float* C_dev,
                                 codenet_report_t* rep_dev, const float* X_next_dev, codenet_stream_t stream,
-                                const LossFuse* fuse) {
+                                const LossFuse* fuse, const PairWish* pair, bool* paired) {
   if (!L || !Delta_dev || !X_dev || B < 1 || B > L->batch_max) return CODENET_E_BADARG;
+  if (paired) *paired = false;
+  L->pair_x = nullptr;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const Geom& g = L->g;
   // the operand copies of the fused tensor-core kernel ride on the vector encoding
@@ -414,8 +462,7 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
   CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit, L->small.on ? &L->small : nullptr));
   int src_kind;
   if (B <= 8) {
-    const bool next = X_next_dev != nullptr && L->next_ok &&
-                      (reinterpret_cast<uintptr_t>(X_next_dev) & 15u) == 0 && (g.n_in % 4) == 0;
+    const bool next = lookahead_ok(L, X_next_dev, B);
     CN_TRY(launch_backward_update_fused(*L, B, lr, L->ws.Y, next ? X_next_dev : nullptr, g.n_in, L->ws.Ynext, st));
     L->next_x = next ? X_next_dev : nullptr;
     L->next_B = B;
@@ -433,6 +480,20 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
   }
   FaultDev fd;
   const bool inject = fill_fault(fault, &fd);
+  if (pair != nullptr && L->next_x != nullptr && C_dev != nullptr && pair->S_next != nullptr && pair_supported(*L, B)) {
+    FaultDev fdn;
+    const bool inject_next = fill_fault(pair->fault_next, &fdn);
+    PairNext nx;
+    nx.X_next = X_next_dev; nx.fault = inject_next ? &fdn : nullptr; nx.S_next = pair->S_next; nx.rep_next = pair->rep_next;
+    nx.commit_S = pair->commit_S; nx.commit_S_to = pair->commit_S_to; nx.commit_n = pair->commit_n;
+    nx.commit_rep = pair->commit_rep; nx.commit_rep_to = pair->commit_rep_to;
+    CN_TRY(launch_check_pair(*L, L->ws.Y, L->ws.Yw, Delta_dev, B, inject ? &fd : nullptr, C_dev, lr, rep_dev, nx, st));
+    L->next_x = nullptr;         // the products taken ahead are used up
+    L->pair_x = X_next_dev;
+    L->pair_B = B;
+    if (paired) *paired = true;
+    return CODENET_OK;
+  }
   CN_TRY(launch_check(*L, CODENET_PHASE_BWD, L->ws.Y, src_kind, L->ws.Yw, Delta_dev, B, inject ? &fd : nullptr, 1, 0,
                       C_dev, lr, 1, rep_dev, st));
   return CODENET_OK;
@@ -446,6 +507,7 @@ int codenet_corrupt_block(codenet_layer_t* L, int i, int j, uint32_t seed, uint3
   CN_TRY(launch_corrupt_block(g, i, j, seed, fault_layer, iteration, density_q32, amplitude,
                               reinterpret_cast<cudaStream_t>(stream)));
   L->next_x = nullptr;   // products taken ahead from the blocks as they were no longer describe them
+  L->pair_x = nullptr;
   return CODENET_OK;
 }
 
@@ -465,6 +527,7 @@ int codenet_regenerate_block(codenet_layer_t* L, int i, int j, int along, codene
   }
   CN_TRY(launch_regenerate_block(g, i, j, along, nullptr, reinterpret_cast<cudaStream_t>(stream)));
   L->next_x = nullptr;
+  L->pair_x = nullptr;
   return CODENET_OK;
 }
 
@@ -534,6 +597,7 @@ int codenet_checkpoint_restore(codenet_layer_t* L, codenet_stream_t stream) {
   CN_TRY(launch_copy_bytes(L->ck_U, L->g.U, ub, st));
   CN_TRY(launch_copy_bytes(L->ck_V, L->g.V, vb, st));
   L->next_x = nullptr;   // products taken ahead from the blocks as they were no longer describe them
+  L->pair_x = nullptr;
   return CODENET_OK;
 }
 
@@ -585,12 +649,16 @@ int codenet_net_create(codenet_layer_t** layers, int L, int activation, int loss
   net->layers.assign(layers, layers + L);
   net->xs.assign(L, nullptr);
   net->out_last = nullptr;
+  net->s_stage = nullptr;
+  net->rep_stage = nullptr;
   net->x_next = nullptr;
   net->delta[0] = net->delta[1] = nullptr;
   net->loss_partials = nullptr;
   cudaError_t e = cudaSuccess;
   for (int l = 1; l < L && e == cudaSuccess; ++l) e = dev_alloc(&net->xs[l], (size_t)bmax * layers[l]->g.n_in);
   if (e == cudaSuccess) e = dev_alloc(&net->out_last, (size_t)bmax * layers[L - 1]->g.n_out);
+  if (e == cudaSuccess && L == 1) e = dev_alloc(&net->s_stage, (size_t)bmax * layers[0]->g.n_out);
+  if (e == cudaSuccess) e = dev_alloc(&net->rep_stage, (size_t)1);
   if (e == cudaSuccess) e = dev_alloc(&net->delta[0], (size_t)bmax * widest);
   if (e == cudaSuccess) e = dev_alloc(&net->delta[1], (size_t)bmax * widest);
   if (e == cudaSuccess) e = dev_alloc(&net->loss_partials, (size_t)513 + LOSS_FUSE_PARTIALS + 1);
@@ -609,6 +677,8 @@ void codenet_free_net(codenet_net_t* net) {
   for (cudaGraphExec_t ge : net->graphs) cudaGraphExecDestroy(ge);
   for (float* p : net->xs) cudaFree(p);
   cudaFree(net->out_last);
+  cudaFree(net->s_stage);
+  cudaFree(net->rep_stage);
   cudaFree(net->delta[0]);
   cudaFree(net->delta[1]);
   cudaFree(net->loss_partials);
@@ -628,8 +698,28 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
   if (!net || !X_dev || !target_dev || B < 1 || B > net->batch_max) return CODENET_E_BADARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const int L = net->L;
+  // The first layer's forward stage may have been done by the previous step (its check shared a launch with that
+  // step's last backward check): its sums are in place (in the staging buffer for a one-layer network), its report
+  // is staged.  And this step may end the same way for the next input.
+  codenet_layer* L0 = net->layers[0];
+  const bool paired_in = L0->pair_x != nullptr && L0->pair_x == X_dev && L0->pair_B == B;
+  const bool pair_out = lookahead_ok(L0, net->x_next, B) && pair_supported(*L0, B);
+  const float* out_cur = net->out_last;   // where this step's last sums are while the step runs
+  PairWish wish;
+  memset(&wish, 0, sizeof(wish));
+  if (paired_in) {
+    codenet_report_t* rep0 = reps_dev ? &reps_dev[0] : nullptr;
+    if (pair_out) {
+      // the paired check at the end of this step copies them out before it reuses the staging buffers
+      if (L == 1) { out_cur = net->s_stage; wish.commit_S = net->s_stage; wish.commit_S_to = net->out_last; wish.commit_n = B * L0->g.n_out; }
+      if (rep0) { wish.commit_rep = net->rep_stage; wish.commit_rep_to = rep0; }
+    } else {
+      if (L == 1) CN_TRY(cudaMemcpyAsync(net->out_last, net->s_stage, (size_t)B * L0->g.n_out * sizeof(float), cudaMemcpyDeviceToDevice, st));
+      if (rep0) CN_TRY(cudaMemcpyAsync(rep0, net->rep_stage, sizeof(codenet_report_t), cudaMemcpyDeviceToDevice, st));
+    }
+  }
   // feedforward: step O1 with its checks, then step C1
-  for (int l = 0; l < L; ++l) {
+  for (int l = paired_in ? 1 : 0; l < L; ++l) {
     const float* x = l == 0 ? X_dev : net->xs[l];
     float* S = l < L - 1 ? net->xs[l + 1] : net->out_last;
     // step C1 rides on the sums: x^{l+1} = f(s^l) is what the check writes
@@ -646,12 +736,12 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
   // (small batches only: with many batch entries the parity segments would form delta m times over)
   const bool fused_loss = net->loss == CODENET_LOSS_MSE_MEAN && n_part <= LOSS_FUSE_PARTIALS && B <= 8;
   if (fused_loss) {
-    fuse.S = net->out_last; fuse.target = reinterpret_cast<const float*>(target_dev); fuse.delta = net->delta[0];
+    fuse.S = out_cur; fuse.target = reinterpret_cast<const float*>(target_dev); fuse.delta = net->delta[0];
     fuse.scale = 1.0f / ((float)gl.n_out * (float)B);
     fuse.partials = net->loss_partials + 513; fuse.counter = reinterpret_cast<unsigned*>(net->loss_partials + 513 + LOSS_FUSE_PARTIALS);
     fuse.loss_out = loss_dev; fuse.n_part = n_part;
   } else {
-    CN_TRY(launch_loss(net->out_last, target_dev, B, gl.n_out, net->loss, net->delta[0], loss_dev,
+    CN_TRY(launch_loss(out_cur, target_dev, B, gl.n_out, net->loss, net->delta[0], loss_dev,
                        net->loss_partials, reinterpret_cast<unsigned*>(net->loss_partials + 512), st));
   }
   // backpropagation: step O2 with its checks fused with the update O3, then step C2
@@ -660,11 +750,28 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
     const float* x = l == 0 ? X_dev : net->xs[l];
     // step C2 rides on the sums: delta^{l-1} = c^l (.) g(x^l)
     net->layers[l]->out_mask = (l > 0 && net->activation == CODENET_ACT_RELU) ? x : nullptr;
+    const bool wish_pair = l == 0 && pair_out;
+    if (wish_pair) {
+      // the forward stage of the next step, first layer: sums to where that step's second layer (or its loss) reads
+      // them, the activation between the layers applied as they are written
+      wish.fault_next = per_layer ? &per_layer[0] : nullptr;
+      wish.S_next = L == 1 ? net->s_stage : net->xs[1];
+      wish.rep_next = net->rep_stage;
+      L0->out_act = L > 1 ? net->activation : CODENET_ACT_IDENTITY;
+    }
+    bool paired = false;
     int rc = backward_update_impl(net->layers[l], net->delta[cur], x, B, lr,
                                   per_layer ? &per_layer[l] : nullptr, net->delta[cur ^ 1],
                                   reps_dev ? &reps_dev[2 * l + 1] : nullptr,
-                                  l == 0 ? net->x_next : nullptr, stream, (l == L - 1 && fused_loss) ? &fuse : nullptr);
+                                  l == 0 ? net->x_next : nullptr, stream, (l == L - 1 && fused_loss) ? &fuse : nullptr,
+                                  wish_pair ? &wish : nullptr, &paired);
     if (rc != CODENET_OK) return rc;
+    if (wish_pair && !paired) {
+      L0->out_act = CODENET_ACT_IDENTITY;
+      // (no pair after all: what was staged for this step goes out by plain copies)
+      if (wish.commit_S) CN_TRY(cudaMemcpyAsync(wish.commit_S_to, wish.commit_S, (size_t)wish.commit_n * sizeof(float), cudaMemcpyDeviceToDevice, st));
+      if (wish.commit_rep) CN_TRY(cudaMemcpyAsync(wish.commit_rep_to, wish.commit_rep, sizeof(codenet_report_t), cudaMemcpyDeviceToDevice, st));
+    }
     cur ^= 1;
   }
   net->x_next = nullptr;

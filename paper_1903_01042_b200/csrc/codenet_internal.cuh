@@ -79,17 +79,21 @@ struct Workspace {
   float* xsum;    // [(j*nsc + s)*B + b] sum of x~_j over the columns of slice s
   float* Y;       // clean un-reduced node outputs (forward) / z partials (backward)
   float* Yw;      // working copy [codeword][node][len][B]
+  float* Yw2;     // the same for the forward part of a paired check (feedforward size), or NULL
+  float* pair_sums;   // paired check: [unit][2] slice sums of the forward part between its phases, or NULL
   float* Ynext;   // feedforward partials of the next iteration [strip][coded row][b], or NULL
   void* tc_x;     // tensor-core operand copy of x: (B, n*ldb) in the multiplication type, or NULL
   void* tc_d;     // tensor-core operand copy of delta~: (B, M*b_r), or NULL
   void* tc_dT;    // transposed operand copies for the update: (M*b_r, B) and (ld, B), or NULL
   void* tc_xT;
   int* tc_flag;   // [0] set by a tensor-core kernel whose bounded wait ran out; [1] which statistics buffer the
-                  // next check kernel works in (kept on the device, flipped by the kernel)
+                  // next check kernel works in (kept on the device, flipped by the kernel); [2] the same for the
+                  // second pair of buffers, those of the forward part of a paired check
   float* chk;     // inner-check scratch for batches > 8 (check_scratch_floats), or NULL
   float* dY;      // output deviations W~_ij nu of nodes whose input copy is hit, [codeword][node][len][B], or NULL
-  CheckStats* stats;  // two buffers used alternately; each check clears the other one
-  CwPlan* plan;       // one per codeword
+  CheckStats* stats;  // two buffers used alternately; each check clears the other one (and two more for the
+                      // forward part of a paired check)
+  CwPlan* plan;       // one per codeword (and a second set for the forward part of a paired check)
   size_t y_elems, yw_elems;
 };
 
@@ -106,6 +110,9 @@ struct codenet_layer {
   int next_ok;               // the layout allows taking the next feedforward products in the update sweep
   const float* next_x;       // input those products were taken for (NULL: none pending)
   int next_B;
+  int pair_ok;               // the buffers of the paired check exist
+  const float* pair_x;       // input whose whole forward stage a paired check has already done (NULL: none)
+  int pair_B;
   // set by codenet_step for the next check of this layer, cleared by it: the activation applied to the
   // forward sums (step C1) and the input whose derivative masks the backward sums (step C2)
   mutable int out_act;
@@ -190,7 +197,23 @@ cudaError_t launch_input_faults(const codenet_layer_impl& L, int B, cudaStream_t
 // Vraw: X (forward) or Delta (backward) as the caller passed it.  commit: write corrected codewords to Yw.
 cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* src, int src_kind, float* Yw,
                          const float* Vraw, int B, const FaultDev* fault, int have_clean, int commit, float* out,
-                         float lr, int update_checksums, codenet_report_t* rep, cudaStream_t st);
+                         float lr, int update_checksums, codenet_report_t* rep, cudaStream_t st, uint32_t it_add = 0u);
+// The backward check of this iteration (arguments as launch_check, phase BWD, partials of the fused sweep) and the
+// forward check of the next one on the products the sweep took ahead (X_next, its fault plan read one iteration
+// on, sums to S_next, report to rep_next) in one cooperative launch.  commit_*: staged sums / report of the previous
+// pair to copy out on entry, or NULL.  The caller has checked pair_supported.
+struct PairNext {
+  const float* X_next;
+  const FaultDev* fault;
+  float* S_next;
+  codenet_report_t* rep_next;
+  const float* commit_S; float* commit_S_to; int commit_n;
+  const codenet_report_t* commit_rep; codenet_report_t* commit_rep_to;
+};
+bool pair_supported(const codenet_layer_impl& L, int B);
+cudaError_t launch_check_pair(const codenet_layer_impl& L, const float* src, float* Yw, const float* Delta, int B,
+                              const FaultDev* fault, float* out, float lr, codenet_report_t* rep,
+                              const PairNext& nx, cudaStream_t st);
 size_t check_scratch_floats(const Geom& g, int B);  // size of Workspace::chk for batches > 8
 cudaError_t launch_sum_outputs(const Geom& g, int phase, int B, const float* Y, float* out, int out_act, codenet_report_t* rep,
                                cudaStream_t st);

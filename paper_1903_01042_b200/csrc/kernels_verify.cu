@@ -336,9 +336,115 @@ __device__ __forceinline__ void big_phase_x_wide(const CheckParams& p, const Pha
   }
 }
 
-template <bool BIG>
-__global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
+// Inner-checksum upkeep for small batches, same rule as the blocks: u += lr (1^T delta~_i) x~_j^T,
+// v += lr delta~_i (x~_j^T 1).  One warp per checksum vector, lanes along it; vectors [vec_begin, vec_end) of the
+// list (all u vectors, then all v vectors), handed out from the last warp of the part backwards.
+__device__ __forceinline__ void update_checksum_vectors(const CheckParams& p, const unsigned bid, const unsigned gdim,
+                                                        int vec_begin, int vec_end) {
+  const Geom& g = p.g;
+  const int B = p.B, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int gw = (gdim - 1 - bid) * CK_WARPS + (CK_WARPS - 1 - warp), nw = gdim * CK_WARPS;
+  const int n_uvec = g.M * g.Nn * g.ns, n_vvec = g.M * g.Nn * g.nsc;
+  for (int vec = vec_begin + gw; vec < vec_end; vec += nw) {
+    const bool is_u = vec < n_uvec;
+    const int v2 = is_u ? vec : vec - n_uvec, nsl = is_u ? g.ns : g.nsc;
+    const int s = v2 % nsl, blk = v2 / nsl;
+    const int i = blk / g.Nn, j = blk % g.Nn;
+    if (i >= g.m && j >= g.n) continue;
+    const int len = is_u ? g.b_c : g.b_r;
+    float* tgt = is_u ? g.U + (size_t)v2 * g.ldb : g.V + (size_t)v2 * g.b_r;
+    // entry e gets lr * sum_b coef[b] * rows[b][e]
+    const float* rows = is_u ? p.Xt + (size_t)j * g.ldb : p.Dt + (size_t)i * g.b_r;
+    const size_t rstride = is_u ? (size_t)g.ld : (size_t)g.Mbr;
+    const float* coef = is_u ? p.dsum + ((size_t)i * g.ns + s) * B : p.xsum + ((size_t)j * g.nsc + s) * B;
+    if ((len & 3) == 0 && (rstride & 3) == 0 &&
+        ((reinterpret_cast<uintptr_t>(tgt) | reinterpret_cast<uintptr_t>(rows)) & 15) == 0) {
+      // 16-byte accesses, eight per lane and round: a 1024-entry vector is one round
+      for (int c0 = 4 * lane; c0 < len; c0 += 128 * 8) {
+        float4 acc[8], old[8];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          const int c = c0 + 128 * w;
+          old[w] = c < len ? *reinterpret_cast<const float4*>(tgt + c) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+          acc[w] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        }
+        for (int b = 0; b < B; ++b) {
+          const float d = coef[b];
+#pragma unroll
+          for (int w = 0; w < 8; ++w) {
+            const int c = c0 + 128 * w;
+            if (c < len) {
+              const float4 x = *reinterpret_cast<const float4*>(rows + (size_t)b * rstride + c);
+              acc[w].x = fmaf(d, x.x, acc[w].x); acc[w].y = fmaf(d, x.y, acc[w].y);
+              acc[w].z = fmaf(d, x.z, acc[w].z); acc[w].w = fmaf(d, x.w, acc[w].w);
+            }
+          }
+        }
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          const int c = c0 + 128 * w;
+          if (c < len)
+            *reinterpret_cast<float4*>(tgt + c) =
+                make_float4(fmaf(p.lr, acc[w].x, old[w].x), fmaf(p.lr, acc[w].y, old[w].y),
+                            fmaf(p.lr, acc[w].z, old[w].z), fmaf(p.lr, acc[w].w, old[w].w));
+        }
+      }
+      continue;
+    }
+    for (int c0 = lane; c0 < len; c0 += 32 * 8) {
+      float acc[8], old[8];
+#pragma unroll
+      for (int w = 0; w < 8; ++w) {  // loads first, so that eight are in flight per lane
+        const int c = c0 + 32 * w;
+        old[w] = c < len ? tgt[c] : 0.0f;
+        acc[w] = 0.0f;
+      }
+      for (int b = 0; b < B; ++b) {
+        const float d = coef[b];
+#pragma unroll
+        for (int w = 0; w < 8; ++w) {
+          const int c = c0 + 32 * w;
+          if (c < len) acc[w] = fmaf(d, rows[(size_t)b * rstride + c], acc[w]);
+        }
+      }
+#pragma unroll
+      for (int w = 0; w < 8; ++w) {
+        const int c = c0 + 32 * w;
+        if (c < len) tgt[c] = fmaf(p.lr, acc[w], old[w]);
+      }
+    }
+  }
+}
+
+// Checksum side of the inner check at batch 1: dot = a . w and dabs = |a| . |w| over lim entries, lanes along the index
+// (each lane's part; the caller adds the lanes up).
+__device__ __forceinline__ void checksum_dot(const float* a, const float* w, int lim, int lane, float& dot, float& dabs) {
+  if ((lim & 3) == 0 && ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(w)) & 15) == 0) {
+    // 16-byte loads: a 1024-entry product is one round of sixteen loads per lane
+#pragma unroll 8
+    for (int c = 4 * lane; c < lim; c += 128) {
+      const float4 av = *reinterpret_cast<const float4*>(a + c), wv = *reinterpret_cast<const float4*>(w + c);
+      dot = fmaf(av.x, wv.x, dot); dabs = fmaf(fabsf(av.x), fabsf(wv.x), dabs);
+      dot = fmaf(av.y, wv.y, dot); dabs = fmaf(fabsf(av.y), fabsf(wv.y), dabs);
+      dot = fmaf(av.z, wv.z, dot); dabs = fmaf(fabsf(av.z), fabsf(wv.z), dabs);
+      dot = fmaf(av.w, wv.w, dot); dabs = fmaf(fabsf(av.w), fabsf(wv.w), dabs);
+    }
+  } else {
+#pragma unroll 16
+    for (int c = lane; c < lim; c += 32) {
+      const float av = a[c], wv = w[c];
+      dot = fmaf(av, wv, dot);
+      dabs = fmaf(fabsf(av), fabsf(wv), dabs);
+    }
+  }
+}
+
+// PAIR: the body runs as one part of a paired launch (p.pair says which); bid / gdim are the CTA's index and the
+// number of CTAs within its part.  Both parts pass the same two grid barriers.
+template <bool BIG, bool PAIR>
+__device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, const unsigned gdim) {
   cg::grid_group grid = cg::this_grid();
+  const bool pair_bwd = PAIR && p.pair == 1, pair_fwd = PAIR && p.pair == 2;
   // which statistics buffer this call works in: read by every CTA before the first grid barrier, flipped by
   // CTA 0 after the second
   const int st_par = __ldcg(p.parity) & 1;
@@ -377,7 +483,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     }
     s_h = h;
   }
-  const uint32_t it = p.fault.iteration ? *p.fault.iteration : 0u;
+  const uint32_t it = (p.fault.iteration ? *p.fault.iteration : 0u) + p.it_add;
   const uint32_t key1 = (p.fault.layer << 8) | (uint32_t)p.phase;
 
   // ------------------------------------------------------------------------------------------
@@ -397,7 +503,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     }
     // units go round the CTAs first and then round the warps, so that a few hundred of them spread over
     // all SMs instead of filling the first CTAs
-    for (int unit = blockIdx.x + gridDim.x * warp; unit < (by_bgroup ? 0 : n_units); unit += gridDim.x * CK_WARPS) {
+    for (int unit = bid + gdim * warp; unit < (by_bgroup ? 0 : n_units); unit += gdim * CK_WARPS) {
       const int s = unit % q.nsl, ck = unit / q.nsl;
       const int k = ck % q.K, cw = ck / q.K;
       const bool hit = (s_inj[cw] >> k) & 1ull, h_out = (s_out[cw] >> k) & 1ull, h_in = (s_in[cw] >> k) & 1ull;
@@ -416,24 +522,8 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
         const float* w = fwd ? p.Vraw + (size_t)j1 * g.b_c : p.Vraw + (size_t)i1 * g.b_r;
         const int lim = fwd ? min(g.b_c, g.n_in - j1 * g.b_c) : min(g.b_r, g.n_out - i1 * g.b_r);
         float dot = 0.0f, dabs = 0.0f, sum_o = 0.0f, sum_abs = 0.0f;
-        if ((lim & 3) == 0 && ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(w)) & 15) == 0) {
-          // 16-byte loads: a 1024-entry product is one round of sixteen loads per lane
-#pragma unroll 8
-          for (int c = 4 * lane; c < lim; c += 128) {
-            const float4 av = *reinterpret_cast<const float4*>(a + c), wv = *reinterpret_cast<const float4*>(w + c);
-            dot = fmaf(av.x, wv.x, dot); dabs = fmaf(fabsf(av.x), fabsf(wv.x), dabs);
-            dot = fmaf(av.y, wv.y, dot); dabs = fmaf(fabsf(av.y), fabsf(wv.y), dabs);
-            dot = fmaf(av.z, wv.z, dot); dabs = fmaf(fabsf(av.z), fabsf(wv.z), dabs);
-            dot = fmaf(av.w, wv.w, dot); dabs = fmaf(fabsf(av.w), fabsf(wv.w), dabs);
-          }
-        } else {
-#pragma unroll 16
-          for (int c = lane; c < lim; c += 32) {
-            const float av = a[c], wv = w[c];
-            dot = fmaf(av, wv, dot);
-            dabs = fmaf(fabsf(av), fabsf(wv), dabs);
-          }
-        }
+        // (the forward part of a pair takes the checksum side after the barrier: the backward part is updating u)
+        if (!pair_fwd) checksum_dot(a, w, lim, lane, dot, dabs);
         // four elements per lane and round, their partials loaded together (clean_value4): a round is a few
         // round trips to memory instead of one per element and sixteen partials
         for (size_t t0 = 0; t0 < SL; t0 += 128) {
@@ -468,7 +558,12 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
         }
         mx = warp_max(mx);
         if (lane == 0) atomicMax(&p.st->norm[cw * MAXN + k], __float_as_uint(mx));
-        sum_o = warp_sum(sum_o); sum_abs = warp_sum(sum_abs); dot = warp_sum(dot); dabs = warp_sum(dabs);
+        sum_o = warp_sum(sum_o); sum_abs = warp_sum(sum_abs);
+        if (pair_fwd) {
+          if (lane == 0) { p.pair_sums[2 * unit] = sum_o; p.pair_sums[2 * unit + 1] = sum_abs; }
+          continue;
+        }
+        dot = warp_sum(dot); dabs = warp_sum(dabs);
         const float ratio = fabsf(sum_o - dot) / (g.tau_rel * dabs + floor_c * sum_abs + g.tau_abs);
         if (lane == 0) atomicMax(&p.st->ratio[cw * MAXN + k], __float_as_uint(ratio));
         continue;
@@ -535,8 +630,8 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       const int n_items = q.n_cw * ugroups * chunks * ncch;
       // handed out from the last warp of the grid backwards: the statistics items above fill the grid from
       // the front, so on small layers the two kinds of work run side by side
-      for (int item = (gridDim.x - 1 - blockIdx.x) * CK_WARPS + (CK_WARPS - 1 - warp); item < n_items;
-           item += gridDim.x * CK_WARPS) {
+      for (int item = (gdim - 1 - bid) * CK_WARPS + (CK_WARPS - 1 - warp); item < n_items;
+           item += gdim * CK_WARPS) {
         const int cc = item % ncch, it3 = item / ncch;
         const int cw = it3 / (ugroups * chunks), rem = it3 % (ugroups * chunks);
         const int u0 = (rem / chunks) * 4, b0 = (rem % chunks) * 8;
@@ -586,14 +681,51 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
       }
     }
   }
+  if (pair_bwd && p.update_checksums) {
+    // the u vectors get this iteration's update before the barrier: the forward part, whose products come from
+    // the updated blocks, reads them after it (nothing in a backward check reads u)
+    update_checksum_vectors(p, bid, gdim, 0, g.M * g.Nn * g.ns);
+  }
+  if (pair_fwd) {
+    // what the forward part of the previous pair left in the staging buffers (sums and report of the iteration
+    // that is ending) goes where the caller reads it, before this part overwrites them behind the barrier
+    if (p.commit_S != nullptr)
+      for (int idx = (int)bid * CK_THREADS + tid; idx < p.commit_n; idx += (int)gdim * CK_THREADS)
+        p.commit_S_to[idx] = p.commit_S[idx];
+    if (p.commit_rep != nullptr && bid == gdim - 1) {
+      const uint32_t* from = reinterpret_cast<const uint32_t*>(p.commit_rep);
+      uint32_t* to = reinterpret_cast<uint32_t*>(p.commit_rep_to);
+      for (int t = tid; t < (int)(sizeof(codenet_report_t) / sizeof(uint32_t)); t += CK_THREADS) to[t] = from[t];
+    }
+  }
   grid.sync();
 
   // ------------------------------------------------------------------------------------------
   // phase X: syndrome maxima; sums assuming no error; inner-checksum update; reset of the
   // statistics buffer of the next call
   // ------------------------------------------------------------------------------------------
-  const size_t gstride = (size_t)gridDim.x * CK_THREADS;
-  const size_t g0 = blockIdx.x * (size_t)CK_THREADS + tid;
+  const size_t gstride = (size_t)gdim * CK_THREADS;
+  const size_t g0 = bid * (size_t)CK_THREADS + tid;
+  if (pair_fwd) {
+    // checksum side of the inner check, u . x, with the u vectors as the backward part has just updated them;
+    // the slice sums wait in pair_sums.  Same units, same warps, same arithmetic as a check of its own.
+    const int n_units = q.n_cw * q.K * q.nsl;
+    const float floor_c = g.tau_rel * (1.0f / 512.0f);
+    for (int unit = bid + gdim * warp; unit < n_units; unit += gdim * CK_WARPS) {
+      const int s = unit % q.nsl, ck = unit / q.nsl;
+      const int k = ck % q.K, cw = ck / q.K;
+      const int blk1 = k * g.Nn + cw;
+      const float* a = g.U + ((size_t)blk1 * g.ns + s) * g.ldb;
+      const float* w = p.Vraw + (size_t)cw * g.b_c;
+      const int lim = min(g.b_c, g.n_in - cw * g.b_c);
+      float dot = 0.0f, dabs = 0.0f;
+      checksum_dot(a, w, lim, lane, dot, dabs);
+      dot = warp_sum(dot); dabs = warp_sum(dabs);
+      const float sum_o = p.pair_sums[2 * unit], sum_abs = p.pair_sums[2 * unit + 1];
+      const float ratio = fabsf(sum_o - dot) / (g.tau_rel * dabs + floor_c * sum_abs + g.tau_abs);
+      if (lane == 0) atomicMax(&p.st->ratio[cw * MAXN + k], __float_as_uint(ratio));
+    }
+  }
   if (big_batch && node_check) {
     const float floor_c = g.tau_rel * (1.0f / 512.0f);
     const size_t total = (size_t)q.n_cw * q.K * q.nsl * B;
@@ -603,8 +735,8 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     // the ratios start behind the CTAs that take the sum tiles below, the checksum update comes from the
     // far end of the grid: three independent pieces of work, side by side on small layers
     const int sum_tiles = ((q.len + BIG_TR - 1) / BIG_TR) * (B / 32);
-    const int rot = sum_tiles % (int)gridDim.x;
-    const size_t g0r = (size_t)((blockIdx.x + gridDim.x - rot) % gridDim.x) * CK_THREADS + tid;
+    const int rot = sum_tiles % (int)gdim;
+    const size_t g0r = (size_t)((bid + gdim - rot) % gdim) * CK_THREADS + tid;
     for (size_t idx = g0r; idx < total; idx += gstride) {
       // partial sums in index order: the same result every run
       const float* c = p.chk + (idx / B) * NS * B + idx % B;   // [unit][partial][b]
@@ -645,8 +777,8 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
   // the far end of the grid, so that the three pieces run side by side instead of one after the other in the
   // first CTAs
   const size_t syn_total = (q.r > 0 && !check_off && !one_pass) ? (size_t)q.n_cw * q.n_el : 0;
-  const unsigned syn_ctas = (unsigned)(((syn_total + CK_THREADS - 1) / CK_THREADS) % gridDim.x);
-  const size_t g0s = (size_t)((blockIdx.x + gridDim.x - syn_ctas) % gridDim.x) * CK_THREADS + tid;
+  const unsigned syn_ctas = (unsigned)(((syn_total + CK_THREADS - 1) / CK_THREADS) % gdim);
+  const size_t g0s = (size_t)((bid + gdim - syn_ctas) % gdim) * CK_THREADS + tid;
   if (q.r > 0 && !check_off && !one_pass) {
     const size_t total = (size_t)q.n_cw * q.n_el;
     for (size_t idx = g0; idx < total; idx += gstride) {
@@ -681,7 +813,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     __shared__ float s_tile[32][33];
     const int nout = fwd ? g.n_out : g.n_in;
     const int tiles_o = (nout + 31) / 32, tiles_b = B / 32;
-    for (int tile = blockIdx.x; tile < tiles_o * tiles_b; tile += gridDim.x) {
+    for (int tile = bid; tile < tiles_o * tiles_b; tile += gdim) {
       const int o0 = (tile / tiles_b) * 32, b0 = (tile % tiles_b) * 32;
 #pragma unroll
       for (int rr = 0; rr < 32 / CK_WARPS; ++rr) {
@@ -724,79 +856,9 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     }
   }
   if (p.update_checksums && !big_batch) {
-    // same rule as the blocks: u += lr (1^T delta~_i) x~_j^T,  v += lr delta~_i (x~_j^T 1).
-    // One warp per checksum vector, lanes along it; handed out from the last warp of the grid backwards.
-    const int gw = (gridDim.x - 1 - blockIdx.x) * CK_WARPS + (CK_WARPS - 1 - warp), nw = gridDim.x * CK_WARPS;
+    // (in a pair the u vectors were updated before the first barrier: the forward part reads them after it)
     const int n_uvec = g.M * g.Nn * g.ns, n_vvec = g.M * g.Nn * g.nsc;
-    for (int vec = gw; vec < n_uvec + n_vvec; vec += nw) {
-      const bool is_u = vec < n_uvec;
-      const int v2 = is_u ? vec : vec - n_uvec, nsl = is_u ? g.ns : g.nsc;
-      const int s = v2 % nsl, blk = v2 / nsl;
-      const int i = blk / g.Nn, j = blk % g.Nn;
-      if (i >= g.m && j >= g.n) continue;
-      const int len = is_u ? g.b_c : g.b_r;
-      float* tgt = is_u ? g.U + (size_t)v2 * g.ldb : g.V + (size_t)v2 * g.b_r;
-      // entry e gets lr * sum_b coef[b] * rows[b][e]
-      const float* rows = is_u ? p.Xt + (size_t)j * g.ldb : p.Dt + (size_t)i * g.b_r;
-      const size_t rstride = is_u ? (size_t)g.ld : (size_t)g.Mbr;
-      const float* coef = is_u ? p.dsum + ((size_t)i * g.ns + s) * B : p.xsum + ((size_t)j * g.nsc + s) * B;
-      if ((len & 3) == 0 && (rstride & 3) == 0 &&
-          ((reinterpret_cast<uintptr_t>(tgt) | reinterpret_cast<uintptr_t>(rows)) & 15) == 0) {
-        // 16-byte accesses, eight per lane and round: a 1024-entry vector is one round
-        for (int c0 = 4 * lane; c0 < len; c0 += 128 * 8) {
-          float4 acc[8], old[8];
-#pragma unroll
-          for (int w = 0; w < 8; ++w) {
-            const int c = c0 + 128 * w;
-            old[w] = c < len ? *reinterpret_cast<const float4*>(tgt + c) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            acc[w] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-          }
-          for (int b = 0; b < B; ++b) {
-            const float d = coef[b];
-#pragma unroll
-            for (int w = 0; w < 8; ++w) {
-              const int c = c0 + 128 * w;
-              if (c < len) {
-                const float4 x = *reinterpret_cast<const float4*>(rows + (size_t)b * rstride + c);
-                acc[w].x = fmaf(d, x.x, acc[w].x); acc[w].y = fmaf(d, x.y, acc[w].y);
-                acc[w].z = fmaf(d, x.z, acc[w].z); acc[w].w = fmaf(d, x.w, acc[w].w);
-              }
-            }
-          }
-#pragma unroll
-          for (int w = 0; w < 8; ++w) {
-            const int c = c0 + 128 * w;
-            if (c < len)
-              *reinterpret_cast<float4*>(tgt + c) =
-                  make_float4(fmaf(p.lr, acc[w].x, old[w].x), fmaf(p.lr, acc[w].y, old[w].y),
-                              fmaf(p.lr, acc[w].z, old[w].z), fmaf(p.lr, acc[w].w, old[w].w));
-          }
-        }
-        continue;
-      }
-      for (int c0 = lane; c0 < len; c0 += 32 * 8) {
-        float acc[8], old[8];
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {  // loads first, so that eight are in flight per lane
-          const int c = c0 + 32 * w;
-          old[w] = c < len ? tgt[c] : 0.0f;
-          acc[w] = 0.0f;
-        }
-        for (int b = 0; b < B; ++b) {
-          const float d = coef[b];
-#pragma unroll
-          for (int w = 0; w < 8; ++w) {
-            const int c = c0 + 32 * w;
-            if (c < len) acc[w] = fmaf(d, rows[(size_t)b * rstride + c], acc[w]);
-          }
-        }
-#pragma unroll
-        for (int w = 0; w < 8; ++w) {
-          const int c = c0 + 32 * w;
-          if (c < len) tgt[c] = fmaf(p.lr, acc[w], old[w]);
-        }
-      }
-    }
+    update_checksum_vectors(p, bid, gdim, pair_bwd ? n_uvec : 0, n_uvec + n_vvec);
   }
   if (p.update_checksums && big_batch && B >= 128) {
     // batches of 128 and more: u_ij += lr sum_b (1^T delta~_i)[b] x~_j[b][:] and
@@ -806,7 +868,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     // a warp takes 32 entries of the rows of one j (or i), up to eight partner blocks and one slice; eight
     // lanes cover the entries, four per lane, and the four lane groups take a quarter of the batch each, added
     // up in a fixed order at the end.
-    const int gw = (gridDim.x - 1 - blockIdx.x) * CK_WARPS + (CK_WARPS - 1 - warp), nw = gridDim.x * CK_WARPS;
+    const int gw = (gdim - 1 - bid) * CK_WARPS + (CK_WARPS - 1 - warp), nw = gdim * CK_WARPS;
     const int uspans = (g.b_c + 31) / 32, vspans = (g.b_r + 31) / 32;
     const int ugr = (g.M + 7) / 8, vgr = (g.Nn + 7) / 8;                      // partner groups
     const int ugs = (g.M + ugr - 1) / ugr, vgs = (g.Nn + vgr - 1) / vgr;      // partners per group, evened out
@@ -895,7 +957,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     // batches under 128: a warp takes 32 entries of one checksum vector (one per lane) and walks the batch in
     // index order, 32 batch entries in flight: one or two rounds of loads per item, and few instructions,
     // which counts on small layers where every warp runs this once
-    const int gw = (gridDim.x - 1 - blockIdx.x) * CK_WARPS + (CK_WARPS - 1 - warp), nw = gridDim.x * CK_WARPS;
+    const int gw = (gdim - 1 - bid) * CK_WARPS + (CK_WARPS - 1 - warp), nw = gdim * CK_WARPS;
     const int ucols = (g.b_c + 31) / 32, vrows = (g.b_r + 31) / 32;
     const int n_blk = g.M * g.Nn;
     const int n_uitems = n_blk * g.ns * ucols, n_vitems = n_blk * g.nsc * vrows;
@@ -932,7 +994,7 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     unsigned* z = reinterpret_cast<unsigned*>(p.st_next);
     for (size_t idx = g0; idx < sizeof(CheckStats) / sizeof(unsigned); idx += gstride) z[idx] = 0u;
   }
-  if (p.rep != nullptr && blockIdx.x == gridDim.x - 1) {
+  if (p.rep != nullptr && bid == gdim - 1) {
     // the report starts empty; every codeword's CTA adds its part in phase D (counts, masks, extremes:
     // all order-independent), so no CTA has to come last and gather
     codenet_report_t* r = p.rep;
@@ -946,12 +1008,12 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     for (int c = q.n_cw + tid; c < MAXN; c += CK_THREADS) { r->flagged_mask[c] = 0ull; r->injected_mask[c] = 0ull; }
   }
   grid.sync();
-  if (blockIdx.x == 0 && tid == 0) *p.parity = st_par ^ 1;
+  if (bid == 0 && tid == 0) *p.parity = st_par ^ 1;
 
   // ------------------------------------------------------------------------------------------
   // phase D: one CTA per codeword decides
   // ------------------------------------------------------------------------------------------
-  for (int cw = blockIdx.x; cw < q.n_cw; cw += gridDim.x) {
+  for (int cw = bid; cw < q.n_cw; cw += gdim) {
     const CwView yw = cw_view(p, q, s_inj, cw);
     const unsigned long long injected = s_inj[cw];
     float cw_min_hit = FLT_MAX, cw_max_clean = 0.0f;
@@ -1222,7 +1284,28 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
     }
   }
   // every CTA read the counter before the first grid barrier
-  if (p.bump != nullptr && blockIdx.x == 0 && tid == 0) *p.bump += 1u;
+  if (p.bump != nullptr && bid == 0 && tid == 0) *p.bump += 1u;
+}
+
+template <bool BIG>
+__global__ void __launch_bounds__(CK_THREADS, 2) check_kernel(CheckParams p) {
+  check_body<BIG, false>(p, blockIdx.x, gridDim.x);
+}
+
+// The backward check of one iteration and the forward check of the next (on the products the update sweep took
+// ahead) in one cooperative launch: CTAs [0, n_first) are the backward part, the rest the forward part, each part
+// with its own statistics buffers, plans, working copy and report.  Small batches only (B = 1, node check, at most
+// one parity per code), where a check is a chain of short latency-bound phases and two of them side by side take
+// little longer than one.
+struct PairParams {
+  CheckParams v[2];
+  int n_first;
+};
+
+__global__ void __launch_bounds__(CK_THREADS, 2) check_pair_kernel(const __grid_constant__ PairParams pp) {
+  const int part = blockIdx.x >= (unsigned)pp.n_first ? 1 : 0;
+  CheckParams p = pp.v[part];
+  check_body<false, true>(p, part ? blockIdx.x - pp.n_first : blockIdx.x, part ? gridDim.x - pp.n_first : pp.n_first);
 }
 
 // SPARE: some plan may have a spare parity to be verified on (two and more parities in the phase's code);
@@ -1436,12 +1519,11 @@ size_t check_scratch_floats(const Geom& g, int B) {
   return worst;
 }
 
-cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* src, int src_kind, float* Yw,
-                         const float* Vraw, int B, const FaultDev* fault, int have_clean, int commit, float* out,
-                         float lr, int update_checksums, codenet_report_t* rep, cudaStream_t st) {
-  cudaError_t e = coop_grid_limits();
-  if (e != cudaSuccess) return e;
-  CheckParams p;
+namespace {
+// Everything of CheckParams that does not depend on how the kernel is launched.
+void fill_check_params(const codenet_layer_impl& L, int phase, const float* src, int src_kind, float* Yw,
+                       const float* Vraw, int B, const FaultDev* fault, int have_clean, int commit, float* out,
+                       float lr, int update_checksums, codenet_report_t* rep, CheckParams& p) {
   p.g = L.g; p.phase = phase; p.B = B; p.src_kind = src_kind; p.have_clean = have_clean; p.RT = L.bwd_rt;
   p.commit = commit; p.update_checksums = update_checksums; p.lr = lr;
   p.spb = L.g.ldb / backward_strip_elems(L.g.dtype);
@@ -1455,6 +1537,70 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
   p.out_act = phase == CODENET_PHASE_FWD ? L.out_act : CODENET_ACT_IDENTITY;
   p.out_mask = phase == CODENET_PHASE_BWD ? L.out_mask : nullptr;
   if (phase == CODENET_PHASE_FWD) L.out_act = CODENET_ACT_IDENTITY; else L.out_mask = nullptr;
+  p.lazy = 0; p.inline_fix = 0; p.bump = nullptr;
+  p.it_add = 0u; p.pair = 0; p.pair_sums = nullptr;
+  p.commit_S = nullptr; p.commit_S_to = nullptr; p.commit_n = 0; p.commit_rep = nullptr; p.commit_rep_to = nullptr;
+}
+}  // namespace
+
+bool pair_supported(const codenet_layer_impl& L, int B) {
+  const Geom& g = L.g;
+  return L.pair_ok && B == 1 && g.locate_mode == CODENET_LOCATE_NODECHECK && g.r_row <= 1 && g.r_col <= 1 &&
+         !L.small.on && keeps_checksums(g);
+}
+
+cudaError_t launch_check_pair(const codenet_layer_impl& L, const float* src, float* Yw, const float* Delta, int B,
+                              const FaultDev* fault, float* out, float lr, codenet_report_t* rep,
+                              const PairNext& nx, cudaStream_t st) {
+  cudaError_t e = coop_grid_limits();
+  if (e != cudaSuccess) return e;
+  const Geom& g = L.g;
+  PairParams pp;
+  memset(&pp, 0, sizeof(pp));
+  CheckParams& pb = pp.v[0];
+  CheckParams& pf = pp.v[1];
+  // (the forward part first: it takes the layer's pending activation, as the forward call it stands for would)
+  fill_check_params(L, CODENET_PHASE_FWD, L.ws.Ynext, 2, L.ws.Yw2, nx.X_next, B, nx.fault, 1, 0, nx.S_next, 0.0f, 0,
+                    nx.rep_next, pf);
+  fill_check_params(L, CODENET_PHASE_BWD, src, 1, Yw, Delta, B, fault, 1, 0, out, lr, 1, rep, pb);
+  pb.pair = 1; pb.inline_fix = 1;
+  pf.pair = 2; pf.inline_fix = 1; pf.it_add = 1u;
+  pf.st_base = L.ws.stats + 2; pf.parity = L.ws.tc_flag + 2; pf.plan = L.ws.plan + CODENET_MAX_NODES;
+  pf.pair_sums = L.ws.pair_sums;
+  pf.commit_S = nx.commit_S; pf.commit_S_to = nx.commit_S_to; pf.commit_n = nx.commit_n;
+  pf.commit_rep = nx.commit_rep; pf.commit_rep_to = nx.commit_rep_to;
+  if (L.bump_after != nullptr) { pb.bump = L.bump_after; L.bump_done = true; }
+  // forward part: one warp per unit and one thread per element; backward part: the same and a warp per checksum
+  // vector, within what is left of the co-resident limit
+  const size_t cap = (size_t)g_coop_blocks_check;
+  size_t nf = ((size_t)g.n * g.M * g.ns + CK_WARPS - 1) / CK_WARPS;
+  const size_t f_el = ((size_t)g.n * g.b_r * B + CK_THREADS - 1) / CK_THREADS;
+  if (f_el > nf) nf = f_el;
+  if (nf > cap / 2) nf = cap / 2;
+  size_t nb = ((size_t)g.m * g.Nn * g.nsc + CK_WARPS - 1) / CK_WARPS;
+  const size_t b_el = ((size_t)g.m * g.b_c * B + CK_THREADS - 1) / CK_THREADS;
+  if (b_el > nb) nb = b_el;
+  const size_t chk = ((size_t)g.M * g.Nn * ((size_t)g.ns * g.ldb + (size_t)g.nsc * g.b_r) + CK_THREADS - 1) / CK_THREADS;
+  if (chk > nb) nb = chk;
+  if (nb > cap - nf) nb = cap - nf;
+  if (nf < 1 || nb < 1) return cudaErrorLaunchOutOfResources;
+  pp.n_first = (int)nb;
+  void* args[] = {&pp};
+  e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(check_pair_kernel), dim3((unsigned)(nb + nf)),
+                                  dim3(CK_THREADS), args, 0, st);
+  if (e != cudaSuccess) return e;
+  count_launch();
+  return cudaSuccess;
+}
+
+cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* src, int src_kind, float* Yw,
+                         const float* Vraw, int B, const FaultDev* fault, int have_clean, int commit, float* out,
+                         float lr, int update_checksums, codenet_report_t* rep, cudaStream_t st, uint32_t it_add) {
+  cudaError_t e = coop_grid_limits();
+  if (e != cudaSuccess) return e;
+  CheckParams p;
+  fill_check_params(L, phase, src, src_kind, Yw, Vraw, B, fault, have_clean, commit, out, lr, update_checksums, rep, p);
+  p.it_add = it_add;
 
   const Geom& g = L.g;
   const bool fwd = phase == CODENET_PHASE_FWD;

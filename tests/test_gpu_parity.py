@@ -594,6 +594,76 @@ def test_next_products_are_dropped_when_another_input_arrives(cn, orc):
     assert _rel(S.cpu().numpy(), p.o.forward(X1)[0]) <= TOL_F32
 
 
+@pytest.mark.parametrize("case", [
+    # n_out, n_in, m, n, rr, rc, B, one launch for the two checks?
+    (1024, 1024, 2, 2, 1, 1, 1, True),
+    (2048, 4096, 4, 8, 1, 1, 1, True),
+    (1024, 2048, 2, 4, 1, 0, 1, True),     # no parity column: the backward codewords carry the node check alone
+    (1024, 1024, 2, 2, 1, 1, 3, False),    # a batch: the two calls one after the other
+    (1024, 1024, 2, 2, 2, 2, 1, False),    # two parities: a decoding plan may need the fix kernel
+    (96, 64, 2, 2, 1, 1, 1, False),        # column strips do not tile the block-columns: no products taken ahead
+])
+def test_backward_update_and_the_next_forward_stage_in_one_call(cn, orc, case):
+    """codenet_backward_update_forward_next against the oracle's backward + update of iteration t followed by its
+    forward stage of iteration t + 1 (fault plan read one iteration on): sums, reports, weights, checksums; and the
+    number of launches says whether the two checks shared one."""
+    no, ni, m, n, rr, rc, B, paired = case
+    W = wl.weights(no, ni, seed=41)
+    p = Pair(cn, orc, W, m, n, rr, rc, batch_max=B)
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rep = cn.new_reports(2)
+    prob = min(0.25, 1.5 / max(m + rr, n + rc))
+    fg = cn.make_fault(seed=43, layer=1, mode=cn.FAULT_BERNOULLI, p=prob, sigma=10.0, iteration_dev=it_dev)
+    fo = orc.make_fault(seed=43, layer=1, mode=orc.FAULT_BERNOULLI, p=prob, sigma=10.0)
+    xs = [_dev(wl.gaussian_inputs(B, ni, seed=44, iteration=it)) for it in range(14)]
+    seen = set()
+    for it in range(13):
+        X = wl.gaussian_inputs(B, ni, seed=44, iteration=it)
+        X1 = wl.gaussian_inputs(B, ni, seed=44, iteration=it + 1)
+        D = wl.gaussian_inputs(B, no, seed=45, iteration=it) / np.float32(B)
+        it_dev.fill_(it)
+        before = cn.launch_count()
+        Cg, Sg = cn.backward_update_forward_next(p.g, _dev(D), xs[it], 0.01, xs[it + 1], fault=fg, fault_next=fg,
+                                                 rep_dev=rep[cn.REPORT_BYTES:], rep_next_dev=rep[:cn.REPORT_BYTES])
+        launches = cn.launch_count() - before
+        Co, rbo = p.o.backward_update(D, X, 0.01, fo, it)
+        So, rfo = p.o.forward(X1, fo, it + 1)
+        rf, rb = cn.read_reports(rep)
+        assert rb.decisions() == rbo.decisions(), ("backward", it)
+        assert rf.decisions() == rfo.decisions(), ("next forward", it)
+        assert _rel(Cg.cpu().numpy(), Co) <= TOL_F32 and _rel(Sg.cpu().numpy(), So) <= TOL_F32
+        for r in (rf, rb):
+            if any(r.injected_mask):
+                assert r.min_margin_hit > 10.0
+            assert r.max_margin_clean < 0.1
+            seen.add(r.status)
+        # vector encoding, fused sweep, one check kernel -- or the separate calls' launches
+        assert (launches == 3) == paired, launches
+    assert cn.CORRECTED in seen and cn.FALLBACK in seen
+    assert _rel(cn.decode_weights(p.g).cpu().numpy(), p.o.decode_weights()) <= 1e-5
+    p.compare_checksums(cn, 1e-5)
+    # a stand-alone forward call afterwards starts from scratch and agrees as well
+    S = cn.forward(p.g, xs[13])
+    assert _rel(S.cpu().numpy(), p.o.forward(wl.gaussian_inputs(B, ni, seed=44, iteration=13))[0]) <= TOL_F32
+
+
+def test_paired_checks_in_a_network_with_hidden_layers(cn, orc):
+    """Three layers with ReLU and the softmax loss, the first with 512-wide blocks (so that its update sweep can take
+    the next products), the next input announced before every step: the first layer's backward check and its next
+    forward check share a launch, the staged report and the activations reach the next step; decisions, outputs
+    and weights as the oracle's."""
+    cfg = wl.Config("mlp", [wl.LayerSpec(384, 2048, 4, 4, 1, 1), wl.LayerSpec(256, 384, 4, 4, 1, 1),
+                            wl.LayerSpec(10, 256, 4, 4, 1, 1)], 1, 0.01, 40,
+                    activation="relu", loss="softmax_ce", inputs="uniform", p=2e-2, seed=5)
+    launches = cn.launch_count()
+    stats = _run_config(cn, orc, cfg, 40, TOL_F32, 1e-4, lookahead=True)
+    with_pairs = cn.launch_count() - launches
+    assert stats["corrected"] > 0
+    launches = cn.launch_count()
+    _run_config(cn, orc, cfg, 40, TOL_F32, 1e-4, lookahead=False)
+    assert with_pairs < cn.launch_count() - launches - 39     # a forward sweep and a check launch fewer per step
+
+
 def test_config2_mlp_relu_softmax(cn, orc):
     """784-1000-1000-10 MLP, 4x4 + 1 + 1 per layer, batch 1; error rate raised so that 200
     iterations see faults in every layer."""
