@@ -304,20 +304,29 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
             results_down(it)
         torch.cuda.synchronize()
     if graphs and not e2e:
-        # one recorded step per input of the pool, in the order they will be replayed; the iteration
-        # counter is a single device word that every recorded step advances
+        # the pool's steps recorded into one graph, in the order they will run (one graph launch per `pool` steps:
+        # no pause between the steps of a replay); the iteration counter is a single device word that every
+        # recorded step advances
         it_ctr = torch.full((1,), warmup, dtype=torch.int32, device="cuda")
         faults = [cn.make_fault(seed=cfg.seed, layer=l, mode=mode, p=cfg.p, sigma=cfg.sigma, iteration_dev=it_ctr)
                   for l in range(L)]
-        ids = {}
+        order = [(warmup + k) % pool for k in range(pool)]
         before = cn.launch_count()
-        for k in range(pool):
-            it = warmup + k
-            ids[it % pool] = cn.net_capture_step(net, dxs[it % pool], dts[it % pool], cfg.lr, faults=faults,
-                                                 reps_dev=reps, loss_dev=loss_dev,
-                                                 X_next_dev=dxs[(it + 1) % pool] if lookahead else None)
+        gid_all = cn.net_capture_steps(net, [dxs[k] for k in order], [dts[k] for k in order], cfg.lr, faults=faults,
+                                       reps_dev=reps, loss_dev=loss_dev,
+                                       X_next_dev=dxs[order[0]] if lookahead else None)
         net.launches_per_recorded_step = (cn.launch_count() - before) // pool
-        replay = lambda it: cn.net_replay(net, ids[it % pool])
+        tail = steps % pool          # the last steps % pool steps: a shorter recording, replayed once at the end
+        gid_tail = None
+        if tail:
+            gid_tail = cn.net_capture_steps(net, [dxs[k] for k in order[:tail]], [dts[k] for k in order[:tail]], cfg.lr,
+                                            faults=faults, reps_dev=reps, loss_dev=loss_dev,
+                                            X_next_dev=dxs[order[tail]] if lookahead else None)
+
+        def replay(it):
+            k = it - warmup
+            if k % pool == 0:
+                cn.net_replay(net, gid_all if k + pool <= steps else gid_tail)
         torch.cuda.synchronize()
     if sampler is not None:
         sampler.start()

@@ -295,6 +295,17 @@ int codenet_net_set_next_input(codenet_net_t* net, const float* X_next_dev);
 int codenet_net_capture_step(codenet_net_t* net, const float* X_dev, const void* target_dev, int B, float lr,
                              const codenet_fault_t* per_layer, codenet_report_t* reps_dev, float* loss_dev,
                              const float* X_next_dev, codenet_stream_t stream, int* graph_id);
+
+/* Record n_steps consecutive codenet_step calls into ONE graph (a replay then runs them back to back, without
+ * the pause between two graph launches): step s takes X_devs[s] and target_devs[s] (host arrays of device
+ * pointers), announces X_devs[s + 1] as the next input (X_next_dev after the last step, or NULL), writes its
+ * reports at reps_dev + s * reps_stride (in reports; 0: every step writes the same 2L reports) and its loss at
+ * loss_dev + s * loss_stride.  Everything else as codenet_net_capture_step.  Errors: BADARG. */
+int codenet_net_capture_steps(codenet_net_t* net, int n_steps, const float* const* X_devs,
+                              const void* const* target_devs, int B, float lr,
+                              const codenet_fault_t* per_layer, codenet_report_t* reps_dev, int reps_stride,
+                              float* loss_dev, int loss_stride, const float* X_next_dev,
+                              codenet_stream_t stream, int* graph_id);
 int codenet_net_replay(codenet_net_t* net, int graph_id, codenet_stream_t stream);
 
 /* Copy the last layer's pre-loss output of the most recent codenet_step into out_dev (B, n_L). */

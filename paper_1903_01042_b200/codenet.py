@@ -91,6 +91,8 @@ def lib():
                                                        C.POINTER(Fault), vp, vp, vp]
     L.codenet_net_set_next_input.argtypes = [vp, vp]
     L.codenet_net_capture_step.argtypes = [vp, vp, vp, ip, fl, C.POINTER(Fault), vp, vp, vp, vp, C.POINTER(ip)]
+    L.codenet_net_capture_steps.argtypes = [vp, ip, C.POINTER(vp), C.POINTER(vp), ip, fl, C.POINTER(Fault), vp, ip,
+                                            vp, ip, vp, vp, C.POINTER(ip)]
     L.codenet_net_replay.argtypes = [vp, ip, vp]
     L.codenet_detect_decode.argtypes = [vp, ip, vp, vp, ip, vp, vp]
     L.codenet_net_create.argtypes = [C.POINTER(vp), ip, ip, ip, C.POINTER(vp)]
@@ -126,6 +128,7 @@ def lib():
                  "codenet_decode_weights", "codenet_check_invariance", "codenet_get_block",
                  "codenet_layer_dims", "codenet_net_output", "codenet_get_checksums",
                  "codenet_backward_update_next", "codenet_backward_update_forward_next", "codenet_net_set_next_input", "codenet_net_capture_step",
+                 "codenet_net_capture_steps",
                  "codenet_net_replay", "codenet_corrupt_block", "codenet_regenerate_block",
                  "codenet_checkpoint_save", "codenet_checkpoint_restore"):
         getattr(L, name).restype = ip
@@ -356,6 +359,25 @@ def net_capture_step(net, X_dev, target_dev, lr, faults=None, reps_dev=None, los
     gid = C.c_int(-1)
     _check(lib().codenet_net_capture_step(net.h, _ptr(X_dev), _ptr(target_dev), B, float(lr), farr, _ptr(reps_dev),
                                           _ptr(loss_dev), _ptr(X_next_dev), _stream(), C.byref(gid)))
+    return int(gid.value)
+
+
+def net_capture_steps(net, X_devs, target_devs, lr, faults=None, reps_dev=None, reps_stride=0, loss_dev=None,
+                      loss_stride=0, X_next_dev=None):
+    """codenet_net_capture_steps: record len(X_devs) consecutive steps into one CUDA graph; returns its id."""
+    B = X_devs[0].shape[0]
+    for x in X_devs:
+        _dev_f32(x, (B, net.layers[0].n_in))
+    n = len(X_devs)
+    xs = (C.c_void_p * n)(*[_ptr(x) for x in X_devs])
+    ts = (C.c_void_p * n)(*[_ptr(t) for t in target_devs])
+    farr = None
+    if faults is not None:
+        farr = (Fault * len(net.layers))(*faults)
+    gid = C.c_int(-1)
+    _check(lib().codenet_net_capture_steps(net.h, n, xs, ts, B, float(lr), farr, _ptr(reps_dev), int(reps_stride),
+                                           _ptr(loss_dev), int(loss_stride), _ptr(X_next_dev), _stream(),
+                                           C.byref(gid)))
     return int(gid.value)
 
 

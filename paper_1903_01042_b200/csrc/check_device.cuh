@@ -47,6 +47,7 @@ struct CheckParams {
   float* pair_sums;        // forward part: [unit][2] slice sum and magnitude sum, from phase U to phase X
   const float* commit_S; float* commit_S_to; int commit_n;   // forward part, on entry: sums and report of the
   const codenet_report_t* commit_rep; codenet_report_t* commit_rep_to;   // previous pair go where the caller reads them
+  const float* loss_partials; int loss_n; float* loss_out;   // forward part: partial sums of this step's loss to add up
 };
 
 struct PhaseGeom {

@@ -416,6 +416,7 @@ struct PairWish {
   codenet_report_t* rep_next;
   const float* commit_S; float* commit_S_to; int commit_n;
   const codenet_report_t* commit_rep; codenet_report_t* commit_rep_to;
+  const float* loss_partials; int loss_n; float* loss_out;
 };
 static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, const float* X_dev, int B,
                                 float lr, const codenet_fault_t* fault, float* C_dev,
@@ -487,6 +488,7 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
     nx.X_next = X_next_dev; nx.fault = inject_next ? &fdn : nullptr; nx.S_next = pair->S_next; nx.rep_next = pair->rep_next;
     nx.commit_S = pair->commit_S; nx.commit_S_to = pair->commit_S_to; nx.commit_n = pair->commit_n;
     nx.commit_rep = pair->commit_rep; nx.commit_rep_to = pair->commit_rep_to;
+    nx.loss_partials = pair->loss_partials; nx.loss_n = pair->loss_n; nx.loss_out = pair->loss_out;
     CN_TRY(launch_check_pair(*L, L->ws.Y, L->ws.Yw, Delta_dev, B, inject ? &fd : nullptr, C_dev, lr, rep_dev, nx, st));
     L->next_x = nullptr;         // the products taken ahead are used up
     L->pair_x = X_next_dev;
@@ -731,6 +733,7 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
   // the mean-squared-error loss rides on the vector encoding of the last layer's backward stage (one
   // kernel fewer); other losses, large batches, or more partial sums than the scratch holds, take the loss kernel
   LossFuse fuse;
+  fuse.defer = 0;
   const Geom& gl = net->layers[L - 1]->g;
   const int n_part = gl.m * gl.ns * B;
   // (small batches only: with many batch entries the parity segments would form delta m times over)
@@ -740,6 +743,10 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
     fuse.scale = 1.0f / ((float)gl.n_out * (float)B);
     fuse.partials = net->loss_partials + 513; fuse.counter = reinterpret_cast<unsigned*>(net->loss_partials + 513 + LOSS_FUSE_PARTIALS);
     fuse.loss_out = loss_dev; fuse.n_part = n_part;
+    // a step that ends with a paired check lets that kernel add the loss partials up: the vector encoding sits
+    // between two sweeps and should not wait for its last CTA
+    fuse.defer = (pair_out && loss_dev != nullptr) ? 1 : 0;
+    if (fuse.defer) { wish.loss_partials = fuse.partials; wish.loss_n = n_part; wish.loss_out = loss_dev; }
   } else {
     CN_TRY(launch_loss(out_cur, target_dev, B, gl.n_out, net->loss, net->delta[0], loss_dev,
                        net->loss_partials, reinterpret_cast<unsigned*>(net->loss_partials + 512), st));
@@ -771,6 +778,7 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
       // (no pair after all: what was staged for this step goes out by plain copies)
       if (wish.commit_S) CN_TRY(cudaMemcpyAsync(wish.commit_S_to, wish.commit_S, (size_t)wish.commit_n * sizeof(float), cudaMemcpyDeviceToDevice, st));
       if (wish.commit_rep) CN_TRY(cudaMemcpyAsync(wish.commit_rep_to, wish.commit_rep, sizeof(codenet_report_t), cudaMemcpyDeviceToDevice, st));
+      if (wish.loss_partials) CN_TRY(launch_sum_loss_partials(wish.loss_partials, wish.loss_n, wish.loss_out, st));
     }
     cur ^= 1;
   }
@@ -781,11 +789,19 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
 int codenet_net_capture_step(codenet_net_t* net, const float* X_dev, const void* target_dev, int B, float lr,
                              const codenet_fault_t* per_layer, codenet_report_t* reps_dev, float* loss_dev,
                              const float* X_next_dev, codenet_stream_t stream, int* graph_id) {
-  if (!net || !graph_id) return CODENET_E_BADARG;
+  return codenet_net_capture_steps(net, 1, &X_dev, &target_dev, B, lr, per_layer, reps_dev, 0, loss_dev, 0, X_next_dev,
+                                   stream, graph_id);
+}
+
+int codenet_net_capture_steps(codenet_net_t* net, int n_steps, const float* const* X_devs,
+                              const void* const* target_devs, int B, float lr, const codenet_fault_t* per_layer,
+                              codenet_report_t* reps_dev, int reps_stride, float* loss_dev, int loss_stride,
+                              const float* X_next_dev, codenet_stream_t stream, int* graph_id) {
+  if (!net || !graph_id || n_steps < 1 || !X_devs || !target_devs || reps_stride < 0 || loss_stride < 0)
+    return CODENET_E_BADARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   if (st == nullptr || stream_is_capturing(st)) return CODENET_E_BADARG;  // the default stream cannot record
   CN_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-  net->x_next = X_next_dev;
   // a recorded step ends by advancing each iteration counter its fault plans read (once per counter).  With one
   // counter for the whole network the step's last kernel, the backward check of the first layer, can do it
   // itself; otherwise one-thread kernels follow.
@@ -798,18 +814,24 @@ int codenet_net_capture_step(codenet_net_t* net, const float* X_dev, const void*
     else if (only != ctr) single = false;
   }
   const codenet_layer_impl* first = net->layers[0];
-  first->bump_after = (single && only != nullptr) ? const_cast<uint32_t*>(only) : nullptr;
-  first->bump_done = false;
-  int rc = codenet_step(net, X_dev, target_dev, B, lr, per_layer, reps_dev, loss_dev, stream);
-  const bool bumped = first->bump_done;
-  first->bump_after = nullptr;
-  first->bump_done = false;
-  if (rc == CODENET_OK && per_layer && !bumped) {
-    for (int l = 0; l < net->L && rc == CODENET_OK; ++l) {
-      const uint32_t* ctr = per_layer[l].iteration_dev;
-      bool seen = ctr == nullptr;
-      for (int k = 0; k < l && !seen; ++k) seen = per_layer[k].iteration_dev == ctr;
-      if (!seen && launch_bump_counter(const_cast<uint32_t*>(ctr), st) != cudaSuccess) rc = CODENET_E_CUDA;
+  int rc = CODENET_OK;
+  for (int s = 0; s < n_steps && rc == CODENET_OK; ++s) {
+    net->x_next = s + 1 < n_steps ? X_devs[s + 1] : X_next_dev;
+    first->bump_after = (single && only != nullptr) ? const_cast<uint32_t*>(only) : nullptr;
+    first->bump_done = false;
+    rc = codenet_step(net, X_devs[s], target_devs[s], B, lr, per_layer,
+                      reps_dev ? reps_dev + (size_t)s * reps_stride : nullptr,
+                      loss_dev ? loss_dev + (size_t)s * loss_stride : nullptr, stream);
+    const bool bumped = first->bump_done;
+    first->bump_after = nullptr;
+    first->bump_done = false;
+    if (rc == CODENET_OK && per_layer && !bumped) {
+      for (int l = 0; l < net->L && rc == CODENET_OK; ++l) {
+        const uint32_t* ctr = per_layer[l].iteration_dev;
+        bool seen = ctr == nullptr;
+        for (int k = 0; k < l && !seen; ++k) seen = per_layer[k].iteration_dev == ctr;
+        if (!seen && launch_bump_counter(const_cast<uint32_t*>(ctr), st) != cudaSuccess) rc = CODENET_E_CUDA;
+      }
     }
   }
   cudaGraph_t graph = nullptr;

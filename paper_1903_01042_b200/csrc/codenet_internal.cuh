@@ -181,6 +181,7 @@ struct LossFuse {
   float scale;            // 1 / (N B)
   float* partials; unsigned* counter; float* loss_out;
   int n_part;
+  int defer;              // the partials are added up later in the step (by the paired check that ends it), not here
 };
 // emit: 0 = the fp32 vectors only; 1 = also their transposes (rows, B) for the fused TF32 kernel; 2 = also the
 // bfloat16 copies the fused bf16 kernel reads (delta~ as a hi / lo pair, x~ rounded).  Sets L.operands_ready
@@ -209,6 +210,7 @@ struct PairNext {
   codenet_report_t* rep_next;
   const float* commit_S; float* commit_S_to; int commit_n;
   const codenet_report_t* commit_rep; codenet_report_t* commit_rep_to;
+  const float* loss_partials; int loss_n; float* loss_out;   // a loss whose partial sums wait to be added up, or NULL
 };
 bool pair_supported(const codenet_layer_impl& L, int B);
 cudaError_t launch_check_pair(const codenet_layer_impl& L, const float* src, float* Yw, const float* Delta, int B,
@@ -232,6 +234,7 @@ cudaError_t launch_activation(float* x, size_t n, int act, cudaStream_t st);
 cudaError_t launch_loss(const float* S, const void* target, int B, int n, int loss, float* delta,
                         float* loss_out, float* partials, unsigned* counter, cudaStream_t st);
 cudaError_t launch_bump_counter(uint32_t* counter, cudaStream_t st);
+cudaError_t launch_sum_loss_partials(const float* partials, int n, float* out, cudaStream_t st);
 cudaError_t launch_mask_delta(float* C, const float* x, size_t n, int act, cudaStream_t st);
 
 // ---- device helpers -------------------------------------------------------------------------

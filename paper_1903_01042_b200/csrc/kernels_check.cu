@@ -241,6 +241,10 @@ encode_vectors_kernel(Geom g, const float* __restrict__ X, const float* __restri
   __syncthreads();
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = loss_part;
   __syncthreads();
+  if (lf.defer) {   // a later kernel of the step adds the partials up, in the order used below
+    if (threadIdx.x == 0 && loss_id >= 0) lf.partials[loss_id] = red[0] + red[1] + red[2] + red[3];
+    return;
+  }
   if (threadIdx.x == 0) {
     if (loss_id >= 0) lf.partials[loss_id] = red[0] + red[1] + red[2] + red[3];
     __threadfence();
@@ -546,7 +550,7 @@ cudaError_t launch_encode_vectors(const codenet_layer_impl& L, const float* X, c
   if (nseg == 0) return cudaSuccess;
   LossFuse lf;
   if (fuse) lf = *fuse;
-  else { lf.S = nullptr; lf.target = nullptr; lf.delta = nullptr; lf.scale = 0.0f; lf.partials = nullptr; lf.counter = nullptr; lf.loss_out = nullptr; lf.n_part = 0; }
+  else { lf.S = nullptr; lf.target = nullptr; lf.delta = nullptr; lf.scale = 0.0f; lf.partials = nullptr; lf.counter = nullptr; lf.loss_out = nullptr; lf.n_part = 0; lf.defer = 0; }
   // the 16-byte path needs every length, offset and pointer to be a multiple of four floats
   const bool vec_ok = g.b_c % 4 == 0 && g.b_r % 4 == 0 && g.Tc % 4 == 0 && g.T % 4 == 0 && g.n_in % 4 == 0 &&
                       g.n_out % 4 == 0 && g.Mbr % 4 == 0 && (reinterpret_cast<uintptr_t>(X) & 15u) == 0 &&
@@ -655,6 +659,23 @@ cudaError_t launch_copy_bytes(const void* src, void* dst, size_t bytes, cudaStre
 }
 
 __global__ void bump_counter_kernel(uint32_t* counter) { *counter += 1u; }
+
+// The loss from its partial sums, in the order the vector-encoding kernel uses when it adds them up itself.
+__global__ void __launch_bounds__(128) sum_loss_partials_kernel(const float* __restrict__ partials, int n, float* out) {
+  __shared__ float red[4];
+  float t = 0.0f;
+  for (int idx = threadIdx.x; idx < n; idx += 128) t += partials[idx];
+  t = warp_sum(t);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = t;
+  __syncthreads();
+  if (threadIdx.x == 0) *out = red[0] + red[1] + red[2] + red[3];
+}
+
+cudaError_t launch_sum_loss_partials(const float* partials, int n, float* out, cudaStream_t st) {
+  sum_loss_partials_kernel<<<1, 128, 0, st>>>(partials, n, out);
+  count_launch();
+  return cudaGetLastError();
+}
 
 cudaError_t launch_bump_counter(uint32_t* counter, cudaStream_t st) {
   bump_counter_kernel<<<1, 1, 0, st>>>(counter);

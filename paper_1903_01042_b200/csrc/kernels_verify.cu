@@ -338,12 +338,15 @@ __device__ __forceinline__ void big_phase_x_wide(const CheckParams& p, const Pha
 
 // Inner-checksum upkeep for small batches, same rule as the blocks: u += lr (1^T delta~_i) x~_j^T,
 // v += lr delta~_i (x~_j^T 1).  One warp per checksum vector, lanes along it; vectors [vec_begin, vec_end) of the
-// list (all u vectors, then all v vectors), handed out from the last warp of the part backwards.
+// list (all u vectors, then all v vectors), handed out from the last warp of the part backwards; warps below
+// first_warp of every CTA take none (they have other work in the same phase).
 __device__ __forceinline__ void update_checksum_vectors(const CheckParams& p, const unsigned bid, const unsigned gdim,
-                                                        int vec_begin, int vec_end) {
+                                                        int vec_begin, int vec_end, int first_warp) {
   const Geom& g = p.g;
   const int B = p.B, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int gw = (gdim - 1 - bid) * CK_WARPS + (CK_WARPS - 1 - warp), nw = gdim * CK_WARPS;
+  if (warp < first_warp) return;
+  const int wpc = CK_WARPS - first_warp;
+  const int gw = (gdim - 1 - bid) * wpc + (CK_WARPS - 1 - warp), nw = gdim * wpc;
   const int n_uvec = g.M * g.Nn * g.ns, n_vvec = g.M * g.Nn * g.nsc;
   for (int vec = vec_begin + gw; vec < vec_end; vec += nw) {
     const bool is_u = vec < n_uvec;
@@ -684,7 +687,9 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
   if (pair_bwd && p.update_checksums) {
     // the u vectors get this iteration's update before the barrier: the forward part, whose products come from
     // the updated blocks, reads them after it (nothing in a backward check reads u)
-    update_checksum_vectors(p, bid, gdim, 0, g.M * g.Nn * g.ns);
+    // (warps that had no unit above: the units went round the CTAs first, so these are the same in every CTA)
+    const int unit_warps = (q.n_cw * q.K * q.nsl + (int)gdim - 1) / (int)gdim;
+    update_checksum_vectors(p, bid, gdim, 0, g.M * g.Nn * g.ns, unit_warps < CK_WARPS ? unit_warps : 0);
   }
   if (pair_fwd) {
     // what the forward part of the previous pair left in the staging buffers (sums and report of the iteration
@@ -692,6 +697,18 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
     if (p.commit_S != nullptr)
       for (int idx = (int)bid * CK_THREADS + tid; idx < p.commit_n; idx += (int)gdim * CK_THREADS)
         p.commit_S_to[idx] = p.commit_S[idx];
+    if (p.loss_partials != nullptr && bid == (gdim > 1 ? gdim - 2 : 0)) {
+      // this step's loss, left as partial sums by the vector encoding: added up in that kernel's own order
+      // (128 threads stride the list, lanes, then the four warps)
+      float t = 0.0f;
+      if (tid < 128)
+        for (int idx = tid; idx < p.loss_n; idx += 128) t += __ldcg(&p.loss_partials[idx]);
+      t = warp_sum(t);
+      if (lane == 0) red[warp] = t;
+      __syncthreads();
+      if (tid == 0) *p.loss_out = red[0] + red[1] + red[2] + red[3];
+      __syncthreads();
+    }
     if (p.commit_rep != nullptr && bid == gdim - 1) {
       const uint32_t* from = reinterpret_cast<const uint32_t*>(p.commit_rep);
       uint32_t* to = reinterpret_cast<uint32_t*>(p.commit_rep_to);
@@ -858,7 +875,7 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
   if (p.update_checksums && !big_batch) {
     // (in a pair the u vectors were updated before the first barrier: the forward part reads them after it)
     const int n_uvec = g.M * g.Nn * g.ns, n_vvec = g.M * g.Nn * g.nsc;
-    update_checksum_vectors(p, bid, gdim, pair_bwd ? n_uvec : 0, n_uvec + n_vvec);
+    update_checksum_vectors(p, bid, gdim, pair_bwd ? n_uvec : 0, n_uvec + n_vvec, 0);
   }
   if (p.update_checksums && big_batch && B >= 128) {
     // batches of 128 and more: u_ij += lr sum_b (1^T delta~_i)[b] x~_j[b][:] and
@@ -1540,6 +1557,7 @@ void fill_check_params(const codenet_layer_impl& L, int phase, const float* src,
   p.lazy = 0; p.inline_fix = 0; p.bump = nullptr;
   p.it_add = 0u; p.pair = 0; p.pair_sums = nullptr;
   p.commit_S = nullptr; p.commit_S_to = nullptr; p.commit_n = 0; p.commit_rep = nullptr; p.commit_rep_to = nullptr;
+  p.loss_partials = nullptr; p.loss_n = 0; p.loss_out = nullptr;
 }
 }  // namespace
 
@@ -1569,6 +1587,7 @@ cudaError_t launch_check_pair(const codenet_layer_impl& L, const float* src, flo
   pf.pair_sums = L.ws.pair_sums;
   pf.commit_S = nx.commit_S; pf.commit_S_to = nx.commit_S_to; pf.commit_n = nx.commit_n;
   pf.commit_rep = nx.commit_rep; pf.commit_rep_to = nx.commit_rep_to;
+  pf.loss_partials = nx.loss_partials; pf.loss_n = nx.loss_n; pf.loss_out = nx.loss_out;
   if (L.bump_after != nullptr) { pb.bump = L.bump_after; L.bump_done = true; }
   // forward part: one warp per unit and one thread per element; backward part: the same and a warp per checksum
   // vector, within what is left of the co-resident limit

@@ -903,6 +903,58 @@ def test_recorded_steps_replay_like_plain_steps(cn, orc, lookahead):
     torch.cuda.set_stream(torch.cuda.default_stream())
 
 
+@pytest.mark.parametrize("lookahead", [False, True])
+def test_several_steps_recorded_into_one_graph(cn, orc, lookahead):
+    """Five consecutive steps over a pool of five inputs recorded into one graph (each with its own reports and loss
+    slot), replayed three times after one plain step.  Inside the recording every step knows its successor's input,
+    so the forward stage of steps two to five is done by the step before; with the input after the last step
+    announced as well, that holds across the end of a replay too.  Against the oracle stepping normally."""
+    cfg = wl.Config("one", [wl.LayerSpec(1024, 2048, 2, 4, 1, 1)], 1, 0.01, 16, p=0.1, seed=9)
+    pairs, gnet, onet = _build_net(cn, orc, cfg)
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fg = [cn.make_fault(seed=3, layer=0, mode=cn.FAULT_BERNOULLI, p=cfg.p, sigma=10.0, iteration_dev=it_dev)]
+    fo = [orc.make_fault(seed=3, layer=0, mode=orc.FAULT_BERNOULLI, p=cfg.p, sigma=10.0)]
+    pool = [wl.layer_inputs(cfg, k) for k in range(5)]
+    xs = [_dev(x) for x, _ in pool]
+    ts = [_dev(t) for _, t in pool]
+    reps = cn.new_reports(2 * 5)
+    losses = torch.zeros(5, device="cuda")
+    side = torch.cuda.Stream()                        # the default stream cannot record a graph
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(side)
+    if lookahead:
+        cn.net_set_next_input(gnet, xs[1])
+    cn.step(gnet, xs[0], ts[0], cfg.lr, faults=fg, reps_dev=reps[:2 * cn.REPORT_BYTES], loss_dev=losses[:1])
+    lo, out_o, reps_o = onet.step(pool[0][0], pool[0][1], cfg.lr, fo, 0)
+    assert [r.decisions() for r in cn.read_reports(reps)[:2]] == [r.decisions() for r in reps_o]
+    order = [1, 2, 3, 4, 0]
+    before = cn.launch_count()
+    graph = cn.net_capture_steps(gnet, [xs[k] for k in order], [ts[k] for k in order], cfg.lr, faults=fg,
+                                 reps_dev=reps, reps_stride=2, loss_dev=losses, loss_stride=1,
+                                 X_next_dev=xs[1] if lookahead else None)
+    # encoding, sweep, one check for two stages -- for every step whose successor the recording knows: all five with
+    # the input after the last one announced, else the first step of a replay runs its own forward stage (sweep, check)
+    assert cn.launch_count() - before == (15 if lookahead else 17), cn.launch_count() - before
+    it_dev.fill_(1)
+    seen = set()
+    for r in range(3):
+        cn.net_replay(gnet, graph)
+        rg = cn.read_reports(reps)
+        lg = losses.cpu().numpy()
+        for s, k in enumerate(order):
+            it = 1 + 5 * r + s
+            lo, out_o, reps_o = onet.step(pool[k][0], pool[k][1], cfg.lr, fo, it)
+            assert [x.decisions() for x in rg[2 * s:2 * s + 2]] == [x.decisions() for x in reps_o], it
+            assert abs(float(lg[s]) - lo) <= 1e-4 * max(1.0, abs(lo)), it
+            seen.update(x.status for x in rg[2 * s:2 * s + 2])
+        assert _rel(gnet.output(1).cpu().numpy(), out_o) <= TOL_F32, r
+    assert cn.CORRECTED in seen and cn.FALLBACK in seen
+    assert _rel(cn.decode_weights(pairs[0].g).cpu().numpy(), pairs[0].o.decode_weights()) <= 1e-4
+    pairs[0].compare_checksums(cn, 1e-5)
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(torch.cuda.default_stream())
+
+
 def test_eager_checks_between_replays_of_a_recorded_step(cn, orc):
     """A recorded step, then an odd number of eager checks on the same layer (an evaluation pass with a fault,
     a stand-alone detect / decode), then the recorded step again: every replay must still decide like the
