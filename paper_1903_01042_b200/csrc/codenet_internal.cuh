@@ -120,6 +120,7 @@ struct codenet_layer {
   // a recorded step's iteration counter: the backward check of the step's last layer advances it itself when
   // no other kernel of the step reads it afterwards (bump_done tells the recorder that it did)
   codenet::SmallDev small = {0, 0, 0, 0, 0, 0, 0.0f, nullptr, 0};   // soft errors in the small steps
+  mutable int sweep_reverse = 0;    // direction of the next single-pass update sweep (alternates)
   mutable int operands_ready = 0;   // the vector-encoding kernel has written the tensor-core operand copies
   mutable uint32_t* bump_after = nullptr;
   mutable bool bump_done = false;

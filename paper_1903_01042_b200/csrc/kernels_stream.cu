@@ -130,15 +130,18 @@ template <typename T, int BT, bool NEXT>
 __global__ void __launch_bounds__(BU_THREADS)
 backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __restrict__ Dt, int B,
                        float lr, int R, int RT, float* __restrict__ zpart,
-                       const float* __restrict__ xnext, int ldxn, float* __restrict__ ynext) {
+                       const float* __restrict__ xnext, int ldxn, float* __restrict__ ynext, int reverse) {
   constexpr int VEC = Raw16<T>::N;
   extern __shared__ float sdelta[];  // [rows of the tile][BT], then (NEXT) [rows][4 warps][BT]
   // Tiles are walked column strip by column strip: the parity block-columns first, then the data
   // block-columns from the last to the first, rows top to bottom inside a strip.  The feedforward
   // pass walks the data block-columns first to last, so each pass starts on what the previous one
-  // touched last and finds part of it still in L2.
+  // touched last and finds part of it still in L2.  When this sweep is the only pass of an iteration (it takes
+  // the next feedforward products as well) every other launch walks the tiles in the opposite order (reverse),
+  // for the same reason: the last tiles of one sweep, updated and still in L2, are the first of the next.
   const int n_rowtiles = g.M * RT;
-  const int strip_order = blockIdx.x / n_rowtiles, rowtile = blockIdx.x % n_rowtiles;
+  const int bx = reverse ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+  const int strip_order = bx / n_rowtiles, rowtile = bx % n_rowtiles;
   const int n_strips = gridDim.x / n_rowtiles;
   const int data_strips = (g.n * g.ldb) / (BU_THREADS * VEC);  // strips wholly inside the data columns
   int strip;
@@ -437,11 +440,13 @@ cudaError_t backward_fused_launch(const codenet_layer_impl& L, int B, float lr, 
   const size_t smem = (size_t)L.bwd_rows * bt * sizeof(float) * (NEXT ? 5 : 1);
   const float* Xt = L.ws.Xt;
   const float* Dt = L.ws.Dt;
+  int reverse = 0;
+  if (NEXT) { reverse = L.sweep_reverse; L.sweep_reverse ^= 1; }
   switch (bt) {
-    case 1: backward_update_kernel<T, 1, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext); break;
-    case 2: backward_update_kernel<T, 2, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext); break;
-    case 4: backward_update_kernel<T, 4, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext); break;
-    default: backward_update_kernel<T, 8, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext); break;
+    case 1: backward_update_kernel<T, 1, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
+    case 2: backward_update_kernel<T, 2, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
+    case 4: backward_update_kernel<T, 4, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
+    default: backward_update_kernel<T, 8, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
   }
   count_launch();
   return cudaGetLastError();
