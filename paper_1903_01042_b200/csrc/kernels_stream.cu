@@ -12,17 +12,31 @@ namespace {
 
 template <typename T> struct Raw16 {
   static constexpr int N = Vec16<T>::N;
-  // Every coded block is touched once per pass: evict-first loads and stores measured fastest
-  // (keeping the tail of a pass in L2 with normal-priority accesses was slower on a B200).
+  // Every coded block is touched once per pass: evict-first loads and stores measured fastest.
   __device__ __forceinline__ static uint4 load_stream(const T* p) {
     return __ldcs(reinterpret_cast<const uint4*>(p));
   }
-  __device__ __forceinline__ static void store_stream(T* p, const uint4& v) {
-    __stcs(reinterpret_cast<uint4*>(p), v);
+  // The same with an L2 eviction policy chosen at run time (createpolicy): evict-first for tiles that will not be
+  // touched again before they leave L2, evict-last for the tail of a sweep that the next sweep starts on.
+  __device__ __forceinline__ static uint4 load_policy(const T* p, uint64_t pol) {
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+    return v;
+  }
+  __device__ __forceinline__ static void store_policy(T* p, const uint4& v, uint64_t pol) {
+    asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1, %2, %3, %4}, %5;"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
   }
   __device__ __forceinline__ static void unpack(const uint4& t, float (&v)[N]);
   __device__ __forceinline__ static uint4 pack(const float (&v)[N]);
 };
+__device__ __forceinline__ uint64_t l2_policy(bool keep) {
+  uint64_t pol;
+  if (keep) asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(pol));
+  else asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 template <> __device__ __forceinline__ void Raw16<float>::unpack(const uint4& t, float (&v)[4]) {
   v[0] = __uint_as_float(t.x); v[1] = __uint_as_float(t.y);
   v[2] = __uint_as_float(t.z); v[3] = __uint_as_float(t.w);
@@ -130,7 +144,7 @@ template <typename T, int BT, bool NEXT>
 __global__ void __launch_bounds__(BU_THREADS)
 backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __restrict__ Dt, int B,
                        float lr, int R, int RT, float* __restrict__ zpart,
-                       const float* __restrict__ xnext, int ldxn, float* __restrict__ ynext, int reverse) {
+                       const float* __restrict__ xnext, int ldxn, float* __restrict__ ynext, int reverse, int keep_from) {
   constexpr int VEC = Raw16<T>::N;
   extern __shared__ float sdelta[];  // [rows of the tile][BT], then (NEXT) [rows][4 warps][BT]
   // Tiles are walked column strip by column strip: the parity block-columns first, then the data
@@ -141,6 +155,9 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
   // for the same reason: the last tiles of one sweep, updated and still in L2, are the first of the next.
   const int n_rowtiles = g.M * RT;
   const int bx = reverse ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+  const uint64_t pol = l2_policy((int)blockIdx.x >= keep_from);   // the last CTAs' tiles stay for the next sweep
+  uint64_t pol_keep;   // the partial sums the check kernel reads next
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
   const int strip_order = bx / n_rowtiles, rowtile = bx % n_rowtiles;
   const int n_strips = gridDim.x / n_rowtiles;
   const int data_strips = (g.n * g.ldb) / (BU_THREADS * VEC);  // strips wholly inside the data columns
@@ -231,7 +248,7 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
     uint4 raw[BU_UNROLL];
 #pragma unroll
     for (int u = 0; u < BU_UNROLL; ++u)
-      if (rr0 + u < nrows) raw[u] = Raw16<T>::load_stream(wp + (size_t)(rr0 + u) * g.ld);
+      if (rr0 + u < nrows) raw[u] = Raw16<T>::load_policy(wp + (size_t)(rr0 + u) * g.ld, pol);
     // the previous rows' partials are summed across the warp while these loads are in flight
     if (NEXT && BT <= 2 && fwd_active && rr0 > 0) reduce_rows(yprev, rr0 - BU_UNROLL);
 #pragma unroll
@@ -251,7 +268,7 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
           }
         }
         const uint4 packed = Raw16<T>::pack(wv);
-        Raw16<T>::store_stream(wp + (size_t)(rr0 + u) * g.ld, packed);
+        Raw16<T>::store_policy(wp + (size_t)(rr0 + u) * g.ld, packed, pol);
         if (NEXT && fwd_active) {  // warp-uniform: a warp's columns lie in one block-column
           float wr[VEC];
           Raw16<T>::unpack(packed, wr);  // the stored (rounded) values are what the next pass would read
@@ -288,7 +305,8 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
       if (b >= B) continue;
       const float* q = sy + (rr * 4) * BT + b;
       const float v = ((q[0] + q[BT]) + q[2 * BT]) + q[3 * BT];
-      ynext[((size_t)strip * g.Mbr + (size_t)i * g.b_r + r0 + rr) * B + b] = v;
+      float* yp = &ynext[((size_t)strip * g.Mbr + (size_t)i * g.b_r + r0 + rr) * B + b];
+      asm volatile("st.global.L2::cache_hint.f32 [%0], %1, %2;" :: "l"(yp), "f"(v), "l"(pol_keep) : "memory");
     }
   }
   if (i < g.m) {
@@ -298,7 +316,8 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
         float* zp = zpart + (((size_t)i * RT + rt) * B + b) * g.ld + gc0;
 #pragma unroll
         for (int q = 0; q < VEC / 4; ++q)
-          reinterpret_cast<float4*>(zp)[q] = make_float4(z[b][4 * q], z[b][4 * q + 1], z[b][4 * q + 2], z[b][4 * q + 3]);
+          asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
+                       :: "l"(zp + 4 * q), "f"(z[b][4 * q]), "f"(z[b][4 * q + 1]), "f"(z[b][4 * q + 2]), "f"(z[b][4 * q + 3]), "l"(pol_keep) : "memory");
       }
   }
 }
@@ -441,12 +460,21 @@ cudaError_t backward_fused_launch(const codenet_layer_impl& L, int B, float lr, 
   const float* Xt = L.ws.Xt;
   const float* Dt = L.ws.Dt;
   int reverse = 0;
-  if (NEXT) { reverse = L.sweep_reverse; L.sweep_reverse ^= 1; }
+  int keep_from = (int)grid.x;   // no tile is kept
+  if (NEXT) {
+    reverse = L.sweep_reverse; L.sweep_reverse ^= 1;
+    // the last 48 MB of a sweep stay at normal priority (measured on a B200 against 0, 96 and 160 MB: larger tails
+    // make the sweep itself faster and the step slower, they crowd out what the kernels between two sweeps read)
+    const size_t keep_bytes = (size_t)48 << 20;
+    const size_t cta_bytes = (size_t)L.bwd_rows * BU_THREADS * 16;
+    const size_t keep_ctas = keep_bytes / cta_bytes;
+    keep_from = keep_ctas >= grid.x ? 0 : (int)(grid.x - keep_ctas);
+  }
   switch (bt) {
-    case 1: backward_update_kernel<T, 1, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
-    case 2: backward_update_kernel<T, 2, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
-    case 4: backward_update_kernel<T, 4, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
-    default: backward_update_kernel<T, 8, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse); break;
+    case 1: backward_update_kernel<T, 1, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
+    case 2: backward_update_kernel<T, 2, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
+    case 4: backward_update_kernel<T, 4, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
+    default: backward_update_kernel<T, 8, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
   }
   count_launch();
   return cudaGetLastError();
