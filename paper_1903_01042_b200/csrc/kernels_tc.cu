@@ -183,13 +183,7 @@ tc_products_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_consta
   __shared__ int s_fail;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // BWD: row0 is a column origin, j a block-row.  The forward products walk the coded rows from the top, all
-  // block-columns of a row group together, and end on the last rows: where the fused backward + update sweep,
-  // which walks the block-rows from the last to the first, begins (and it ends where this walk starts), so each
-  // sweep finds the other's last tiles in L2.
-  const int lin = blockIdx.y * gridDim.x + blockIdx.x;
-  const int row0 = (BWD ? (int)blockIdx.x : lin / (int)gridDim.y) * (MT * TC_TILE_M);
-  const int j = BWD ? (int)blockIdx.y : lin % (int)gridDim.y;
+  const int row0 = blockIdx.x * (MT * TC_TILE_M), j = blockIdx.y;  // BWD: row0 is a column origin, j a block-row
   constexpr int elems_per_kstep = TC_KBYTES / (TF32 ? 4 : 2);  // K elements per stage = elements per 128-byte chunk
   constexpr int CH = TC_TILE_M / elems_per_kstep;                 // BWD: 128-byte column chunks per tile
   constexpr uint32_t chunk_bytes = elems_per_kstep * TC_KBYTES;   // BWD: KT rows of 128 bytes
@@ -850,7 +844,6 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
 
   // item -> (block-row, column tile); tiles of the absent corner (parity row x parity column) are not items
   auto item_of = [&](int item, int* i_blk, int* ct) {
-    item = p.n_items - 1 - item;   // from the last block-row to the first (see tc_products_kernel)
     const int data_items = p.g.m * n_ct;
     if (item < data_items) { *i_blk = item / n_ct; *ct = item % n_ct; }
     else {
