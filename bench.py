@@ -256,6 +256,11 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
         hout = houts[0]
         done = [torch.cuda.Event() for _ in range(2)]
         seen = {"loss": 0.0}
+        # (recorded steps: a ring of four staging buffers, see below; the last warm-up step announces its first one)
+        stage3 = [torch.empty(xb + tb, dtype=torch.uint8, device="cuda") for _ in range(4)]
+        sx3 = [st_[:xb].view(hx[0].dtype).view(hx[0].shape) for st_ in stage3]
+        st3 = [st_[xb:].view(ht[0].dtype).view(ht[0].shape) for st_ in stage3]
+        sx3[3].copy_(hx[warmup % pool])                      # the input of the first recorded step
 
         def results_down(it):
             houts[it % 2].copy_(out_dev, non_blocking=True)
@@ -275,7 +280,7 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
             # during the previous one), so that the update sweep can already use the next input
             stage[it % 2].copy_(hs[it % pool], non_blocking=True)
             if lookahead:
-                cn.net_set_next_input(net, sx[it % 2])
+                cn.net_set_next_input(net, sx3[3] if (graphs and it == warmup - 1) else sx[it % 2])
             cn.step(net, sx[(it + 1) % 2], stt[it % 2], cfg.lr, faults=faults, reps_dev=reps, loss_dev=loss_dev)
             results_down(it)
         else:
@@ -288,20 +293,74 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
     torch.cuda.synchronize()
     replay = None
     if graphs and e2e:
-        # end to end with recorded steps: two graphs over the two input buffers; the host copies go around
-        # them on the same stream (next input and target up before the replay, loss and reports down after)
+        # End to end with the steps in a graph of the caller's own: the eight steps of the pool are captured
+        # together WITH their copies, uploads and downloads on streams of their own.  Step k reads its input from
+        # staging buffer (k - 1) % 4 (it went up for step k - 1) and its target and the next input from buffer
+        # k % 4, which may go up as soon as step k - 3, its last reader, has ended; every step has its own result
+        # slot, copied down behind it.  The host reads a replay's eight losses from pinned memory after it has queued
+        # the next replay.  The network advances the fault plans' iteration counter itself.
         it_ctr = torch.full((1,), warmup, dtype=torch.int32, device="cuda")
         faults = [cn.make_fault(seed=cfg.seed, layer=l, mode=mode, p=cfg.p, sigma=cfg.sigma, iteration_dev=it_ctr)
                   for l in range(L)]
-        gid = {}
-        for k in (warmup % 2, 1 - warmup % 2):      # in the order of the replays: each recording continues
-            gid[k] = cn.net_capture_step(net, sx[1 - k], stt[k], cfg.lr, faults=faults, reps_dev=reps, loss_dev=loss_dev,
-                                         X_next_dev=sx[k] if lookahead else None)   # the look-ahead state
+        cn.net_set_iteration_counter(net, it_ctr)
+        slot = rb + 16
+        outs_dev = torch.zeros(pool * slot, dtype=torch.uint8, device="cuda")
+        outs_host = [torch.empty(pool * slot, dtype=torch.uint8).pin_memory() for _ in range(2)]
+        order = [(warmup + k) % pool for k in range(pool)]
+        main, up, down = torch.cuda.current_stream(), torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+
+        def record(dst_host, n_rec):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=main):
+                step_done = []
+                up.wait_stream(main)
+                down.wait_stream(main)
+                for k in range(n_rec):
+                    src = order[k]
+                    if k >= 3:
+                        up.wait_event(step_done[k - 3])
+                    with torch.cuda.stream(up):
+                        stage3[k % 4].copy_(hs[src], non_blocking=True)      # [x of step k + 1 | target of step k]
+                    main.wait_stream(up)
+                    o = outs_dev[k * slot:(k + 1) * slot]
+                    if lookahead:
+                        cn.net_set_next_input(net, sx3[k % 4])
+                    cn.step(net, sx3[(k - 1) % 4], st3[k % 4], cfg.lr, faults=faults, reps_dev=o[:rb],
+                            loss_dev=o[rb:rb + 4].view(torch.float32))
+                    ev = torch.cuda.Event()
+                    ev.record(main)
+                    step_done.append(ev)
+                    down.wait_event(ev)
+                    with torch.cuda.stream(down):
+                        dst_host[k * slot:(k + 1) * slot].copy_(o, non_blocking=True)
+                main.wait_stream(up)
+                main.wait_stream(down)
+            return g
+        before = cn.launch_count()
+        # recorded in the order of the replays (each recording continues the look-ahead state of the one before):
+        # whole pools alternating between the two host buffers, then the last steps % pool steps once
+        n_full, tail = steps // pool, steps % pool
+        graphs2 = [record(outs_host[r], pool) for r in range(min(n_full, 2))]
+        net.launches_per_recorded_step = (cn.launch_count() - before) // max(1, pool * len(graphs2))
+        g_tail = record(outs_host[n_full % 2], tail) if tail else None
+        if not graphs2:
+            net.launches_per_recorded_step = (cn.launch_count() - before) // tail
+        done = [torch.cuda.Event() for _ in range(2)]
+        seen = {"loss": 0.0}
+        hout = outs_host[0][:slot]
 
         def replay(it):
-            stage[it % 2].copy_(hs[it % pool], non_blocking=True)
-            cn.net_replay(net, gid[it % 2])
-            results_down(it)
+            k = it - warmup
+            if k % pool:
+                return
+            r = k // pool
+            (graphs2[r % 2] if r < n_full else g_tail).replay()
+            done[r % 2].record()
+            if r > 0:
+                done[(r - 1) % 2].synchronize()
+                for q in range(pool):                        # the caller's read of every step's loss
+                    seen["loss"] = float(outs_host[(r - 1) % 2][q * slot + rb:q * slot + rb + 4].view(torch.float32)[0])
         torch.cuda.synchronize()
     if graphs and not e2e:
         # the pool's steps recorded into one graph, in the order they will run (one graph launch per `pool` steps:
@@ -346,6 +405,7 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
     bytes_in = int(hs[0].numel()) if e2e else 0
     bytes_out = int(hout.numel()) if e2e else 0
     launched = cn.launch_count() - launches0
+    cn.net_set_iteration_counter(net, None)
     if replay is not None:
         launched = steps * getattr(net, "launches_per_recorded_step", 0)
     return secs, launched, bytes_in, bytes_out
@@ -589,9 +649,13 @@ def main():
         line["e2e"] = {"value": whole_job_value(world, args.steps, L, max_over_ranks(e_secs, world)),
                        "unit": "layer-iterations/s",
                        "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo,
-                       "note": "every step: one pinned upload of [next input | target], the recorded step, one download "
-                               "of [reports | loss]; the host reads step k - 1's loss from pinned memory after it has "
-                               "queued step k (one step of lag, so the device does not wait for the host's launches)"}
+                       "note": "every step: one pinned upload of [next input | target], the step, one download of "
+                               "[reports | loss]; eight steps and their copies are captured in one graph of the "
+                               "caller's (uploads and downloads on streams of their own), the host reads a replay's "
+                               "losses from pinned memory after it has queued the next replay"
+                               if not args.no_graphs else
+                               "every step: one pinned upload of [next input | target], the step, one download of "
+                               "[reports | loss]; the host reads step k - 1's loss after it has queued step k"}
     if rank == 0 and not args.no_extras:
         # ---- regeneration of a stored block from the code of its block-column: one launch per block, walking
         # the data grid so that every launch reads blocks the previous ones did not leave in L2 ----

@@ -282,6 +282,12 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
  * its sums and report appear where this interface says when that step ends).  One-shot: cleared by that step. */
 int codenet_net_set_next_input(codenet_net_t* net, const float* X_next_dev);
 
+/* Give the network an iteration counter of its own (a device word, e.g. the one the fault plans read): every
+ * codenet_step from now on ends by adding one to it, in its last kernel where that kernel can (so a step the caller
+ * captures into a graph of their own draws a new fault pattern at every replay, like the recorded steps below).
+ * NULL switches it off.  Errors: BADARG. */
+int codenet_net_set_iteration_counter(codenet_net_t* net, uint32_t* counter_dev);
+
 /* Record one codenet_step (same arguments; X_next_dev as in codenet_net_set_next_input, or NULL) into a
  * CUDA graph instead of running it, and keep the instantiated graph in the network; *graph_id names it.
  * Nothing is computed by this call.  `stream` must be a created stream, not the default stream

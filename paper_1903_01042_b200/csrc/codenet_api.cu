@@ -16,6 +16,7 @@ struct codenet_net {
   const float* x_next;     // input of the next step, for layer 1's look-ahead products (one-shot)
   float* s_stage;          // one-layer networks: sums of the next step's forward stage, done ahead by a paired check
   codenet_report_t* rep_stage;   // its report, until the step it belongs to ends
+  uint32_t* step_counter;  // device word every codenet_step advances when it ends (codenet_net_set_iteration_counter), or NULL
   float* delta[2];         // ping-pong error vectors, (B, widest layer)
   float* loss_partials;    // 512 partial sums + one counter word (loss kernel), then LOSS_FUSE_PARTIALS + a counter (loss folded into the vector encoding)
   std::vector<cudaGraphExec_t> graphs;  // captured steps (codenet_net_capture_step)
@@ -653,6 +654,7 @@ int codenet_net_create(codenet_layer_t** layers, int L, int activation, int loss
   net->out_last = nullptr;
   net->s_stage = nullptr;
   net->rep_stage = nullptr;
+  net->step_counter = nullptr;
   net->x_next = nullptr;
   net->delta[0] = net->delta[1] = nullptr;
   net->loss_partials = nullptr;
@@ -751,6 +753,10 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
     CN_TRY(launch_loss(out_cur, target_dev, B, gl.n_out, net->loss, net->delta[0], loss_dev,
                        net->loss_partials, reinterpret_cast<unsigned*>(net->loss_partials + 512), st));
   }
+  // a step counter of the network's own: the step's last check kernel advances it where it can (a recording sets
+  // bump_after itself and then this stays out of the way)
+  const bool own_bump = net->step_counter != nullptr && L0->bump_after == nullptr;
+  if (own_bump) { L0->bump_after = net->step_counter; L0->bump_done = false; }
   // backpropagation: step O2 with its checks fused with the update O3, then step C2
   int cur = 0;
   for (int l = L - 1; l >= 0; --l) {
@@ -783,6 +789,18 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
     cur ^= 1;
   }
   net->x_next = nullptr;
+  if (own_bump) {
+    const bool bumped = L0->bump_done;
+    L0->bump_after = nullptr;
+    L0->bump_done = false;
+    if (!bumped) CN_TRY(launch_bump_counter(net->step_counter, st));
+  }
+  return CODENET_OK;
+}
+
+int codenet_net_set_iteration_counter(codenet_net_t* net, uint32_t* counter_dev) {
+  if (!net) return CODENET_E_BADARG;
+  net->step_counter = counter_dev;
   return CODENET_OK;
 }
 

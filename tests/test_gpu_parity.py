@@ -955,6 +955,72 @@ def test_several_steps_recorded_into_one_graph(cn, orc, lookahead):
     torch.cuda.set_stream(torch.cuda.default_stream())
 
 
+def test_steps_in_a_graph_of_the_callers_own_with_copies_around_them(cn, orc):
+    """The caller captures four steps into a CUDA graph of their own, each with the upload of its target and next
+    input from pinned host memory (on a second stream) and the download of its reports and loss; the network
+    advances the fault plans' iteration counter itself (codenet_net_set_iteration_counter).  Three replays with the
+    host buffers refilled in between, against the oracle stepping normally."""
+    cfg = wl.Config("one", [wl.LayerSpec(1024, 2048, 2, 4, 1, 1)], 1, 0.01, 16, p=0.1, seed=11)
+    pairs, gnet, onet = _build_net(cn, orc, cfg)
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fg = [cn.make_fault(seed=3, layer=0, mode=cn.FAULT_BERNOULLI, p=cfg.p, sigma=10.0, iteration_dev=it_dev)]
+    fo = [orc.make_fault(seed=3, layer=0, mode=orc.FAULT_BERNOULLI, p=cfg.p, sigma=10.0)]
+    n_steps, n_in, n_out = 4, 2048, 1024
+    inputs = [wl.layer_inputs(cfg, it) for it in range(3 * n_steps + 1)]
+    # host side: per step [next input | target]; device side: a ring of four staging buffers
+    h_up = [torch.empty(n_in + n_out).pin_memory() for _ in range(n_steps)]
+    stage = [torch.zeros(n_in + n_out, device="cuda") for _ in range(4)]
+    sx = [b[:n_in].view(1, n_in) for b in stage]
+    st = [b[n_in:].view(1, n_out) for b in stage]
+    slot = 2 * cn.REPORT_BYTES + 16
+    out_dev = torch.zeros(n_steps * slot, dtype=torch.uint8, device="cuda")
+    h_out = torch.empty(n_steps * slot, dtype=torch.uint8).pin_memory()
+    main, up = torch.cuda.Stream(), torch.cuda.Stream()
+    cn.net_set_iteration_counter(gnet, it_dev)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(main):
+        sx[3].copy_(_dev(inputs[0][0]))                      # the input of step 0, as if uploaded for the step before
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=main):
+            up.wait_stream(main)
+            step_done = []
+            for k in range(n_steps):
+                if k >= 3:
+                    up.wait_event(step_done[k - 3])          # buffer k % 4 held the input of step k - 3
+                with torch.cuda.stream(up):
+                    stage[k % 4].copy_(h_up[k], non_blocking=True)
+                main.wait_stream(up)
+                o = out_dev[k * slot:(k + 1) * slot]
+                cn.net_set_next_input(gnet, sx[k % 4])
+                cn.step(gnet, sx[(k - 1) % 4], st[k % 4], cfg.lr, faults=fg, reps_dev=o[:2 * cn.REPORT_BYTES],
+                        loss_dev=o[2 * cn.REPORT_BYTES:2 * cn.REPORT_BYTES + 4].view(torch.float32))
+                h_out[k * slot:(k + 1) * slot].copy_(o, non_blocking=True)
+                step_done.append(torch.cuda.Event())
+                step_done[-1].record(main)
+        seen = set()
+        for r in range(3):
+            for k in range(n_steps):
+                it = r * n_steps + k
+                h_up[k][:n_in].copy_(torch.tensor(inputs[it + 1][0]).reshape(-1))
+                h_up[k][n_in:].copy_(torch.tensor(inputs[it][1]).reshape(-1))
+            graph.replay()
+            main.synchronize()
+            assert int(it_dev.item()) == (r + 1) * n_steps       # the network advanced the counter, once per step
+            for k in range(n_steps):
+                it = r * n_steps + k
+                lo, out_o, reps_o = onet.step(inputs[it][0], inputs[it][1], cfg.lr, fo, it)
+                rg = cn.read_reports(h_out[k * slot:k * slot + 2 * cn.REPORT_BYTES])
+                assert [x.decisions() for x in rg] == [x.decisions() for x in reps_o], it
+                loss = float(h_out[k * slot + 2 * cn.REPORT_BYTES:k * slot + 2 * cn.REPORT_BYTES + 4].view(torch.float32)[0])
+                assert abs(loss - lo) <= 1e-4 * max(1.0, abs(lo)), it
+                seen.update(x.status for x in rg)
+            assert _rel(gnet.output(1).cpu().numpy(), out_o) <= TOL_F32, r
+        assert cn.CORRECTED in seen
+        assert _rel(cn.decode_weights(pairs[0].g).cpu().numpy(), pairs[0].o.decode_weights()) <= 1e-4
+    cn.net_set_iteration_counter(gnet, None)
+    torch.cuda.synchronize()
+
+
 def test_eager_checks_between_replays_of_a_recorded_step(cn, orc):
     """A recorded step, then an odd number of eager checks on the same layer (an evaluation pass with a fault,
     a stand-alone detect / decode), then the recorded step again: every replay must still decide like the
