@@ -74,6 +74,23 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y) : "memory");
 }
+// The same with an L2 eviction policy (createpolicy): the coded weights stream through once per kernel, evict-first
+// keeps them from pushing out what is read again and again (the operand tiles, the node outputs the check kernel reads
+// next, and the instructions of the kernels that follow, which live in the same cache).
+__device__ __forceinline__ uint64_t l2_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_2d_hint(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+      ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(x), "r"(y), "l"(pol) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d_hint(const CUtensorMap* map, int x, int y, const void* src, uint64_t pol) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
+               ::"l"(map), "r"(smem_u32(src)), "r"(x), "r"(y), "l"(pol) : "memory");
+}
 // Tile from shared memory back to global memory (bulk group of the issuing thread).
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, const void* src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
@@ -204,6 +221,7 @@ tc_products_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_consta
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----
+    const uint64_t w_pol = l2_evict_first();
     for (int k = 0; k < (c_withhold_loads ? 0 : p.ksteps); ++k) {
       const int s = k % STAGES;
       if (k >= STAGES && !mbar_wait(&empty[s], ((k / STAGES) - 1) & 1)) { s_fail = 1; break; }
@@ -211,7 +229,7 @@ tc_products_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_consta
       if (!BWD) {
         const int x = j * p.g.ldb + k * elems_per_kstep;
 #pragma unroll
-        for (int t = 0; t < MT; ++t) tma_load_2d(sA + (size_t)s * a_bytes + t * a_tile, &mapW, x, row0 + t * TC_TILE_M, &full[s]);
+        for (int t = 0; t < MT; ++t) tma_load_2d_hint(sA + (size_t)s * a_bytes + t * a_tile, &mapW, x, row0 + t * TC_TILE_M, &full[s], w_pol);
 #pragma unroll
         for (int h = 0; h < SPLIT; ++h) tma_load_2d(sB + (size_t)s * b_bytes + h * b_tile, &mapX, x, h * N, &full[s]);
       } else {
@@ -220,8 +238,8 @@ tc_products_kernel(const __grid_constant__ CUtensorMap mapW, const __grid_consta
         for (int t = 0; t < MT; ++t)
 #pragma unroll
           for (int ch = 0; ch < CH; ++ch)
-            tma_load_2d(sA + (size_t)s * a_bytes + t * a_tile + ch * chunk_bytes, &mapW,
-                        row0 + t * TC_TILE_M + ch * elems_per_kstep, y, &full[s]);
+            tma_load_2d_hint(sA + (size_t)s * a_bytes + t * a_tile + ch * chunk_bytes, &mapW,
+                             row0 + t * TC_TILE_M + ch * elems_per_kstep, y, &full[s], w_pol);
 #pragma unroll
         for (int h = 0; h < SPLIT; ++h) tma_load_2d(sB + (size_t)s * b_bytes + h * b_tile, &mapX, y, h * N, &full[s]);
       }
@@ -855,6 +873,7 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
 
   if (warp == 0 && lane == 0) {
     // ---- TMA producer ----
+    const uint64_t w_pol = l2_evict_first();
     uint32_t wn = 0, dn = 0, xn = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++xn) {
@@ -868,7 +887,7 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
         mbar_expect_tx(&w_full[s], TCF_WTILE);
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch)
-          tma_load_2d(sW + (size_t)s * TCF_WTILE + ch * WCHUNK, &mapW, ct * TC_TILE_M + ch * EPC, row0, &w_full[s]);
+          tma_load_2d_hint(sW + (size_t)s * TCF_WTILE + ch * WCHUNK, &mapW, ct * TC_TILE_M + ch * EPC, row0, &w_full[s], w_pol);
         for (int part = 0; part < (need_z ? Cfg::PARTS : 1); ++part, ++dn) {   // delta~ (hi, then lo)
           const uint32_t ds = dn % TCF_DST;
           if (dn >= TCF_DST && !mbar_wait(&d_empty[ds], ((dn / TCF_DST) - 1) & 1)) { ok = false; break; }
@@ -1054,6 +1073,7 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
     if (!alive) s_fail = 1;
   } else if (warp == 10 && lane == 0) {
     // ---- store warp: a tile every epilogue warp has finished goes back to global memory ----
+    const uint64_t w_pol = l2_evict_first();
     uint32_t wn = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
@@ -1065,7 +1085,7 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
         const int row0 = i_blk * p.g.b_r + rt * TC_TILE_M;
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch)
-          tma_store_2d(&mapW, ct * TC_TILE_M + ch * EPC, row0, sW + (size_t)s * TCF_WTILE + ch * WCHUNK);
+          tma_store_2d_hint(&mapW, ct * TC_TILE_M + ch * EPC, row0, sW + (size_t)s * TCF_WTILE + ch * WCHUNK, w_pol);
         tma_store_commit();
         tma_store_wait_read();
         mbar_arrive(&w_empty[s]);
