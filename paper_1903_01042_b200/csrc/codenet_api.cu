@@ -461,7 +461,10 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
   const Geom& g = L->g;
   // the operand copies of the fused tensor-core kernel ride on the vector encoding
   const int emit = (B > 8 && tc_backward_update_supported(g, L->desc.math, B)) ? (g.dtype == CODENET_F32 ? 1 : 2) : 0;
-  CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit, L->small.on ? &L->small : nullptr));
+  // (a fused tensor-core sweep that shares items out among CTAs adds into Z: the encoding kernel clears it on its way)
+  const bool clear_z = emit != 0 && tc_backward_update_splits(*L, B);
+  CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit, L->small.on ? &L->small : nullptr,
+                               clear_z ? L->ws.Y : nullptr, clear_z ? (size_t)g.m * g.Nn * g.b_c * B : 0));
   int src_kind;
   if (B <= 8) {
     const bool next = lookahead_ok(L, X_next_dev, B);

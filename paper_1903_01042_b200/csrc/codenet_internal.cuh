@@ -120,6 +120,7 @@ struct codenet_layer {
   // a recorded step's iteration counter: the backward check of the step's last layer advances it itself when
   // no other kernel of the step reads it afterwards (bump_done tells the recorder that it did)
   codenet::SmallDev small = {0, 0, 0, 0, 0, 0, 0.0f, nullptr, 0};   // soft errors in the small steps
+  mutable int z_cleared = 0;        // the vector-encoding kernel has zeroed the backward outputs for the split sweep
   mutable int sweep_reverse = 0;    // direction of the next single-pass update sweep (alternates)
   mutable int operands_ready = 0;   // the vector-encoding kernel has written the tensor-core operand copies
   mutable uint32_t* bump_after = nullptr;
@@ -190,7 +191,9 @@ struct LossFuse {
 // small != NULL: soft errors in the additional encoding (the parity sub-vectors of hit units get noise)
 cudaError_t launch_encode_vectors(const codenet_layer_impl& L, const float* X, const float* Delta,
                                   int B, cudaStream_t st, const LossFuse* fuse = nullptr, int emit = 0,
-                                  const SmallDev* small = nullptr);
+                                  const SmallDev* small = nullptr, float* clear = nullptr, size_t clear_floats = 0);
+// Does the fused tensor-core sweep share an item's row tiles out among two CTAs (which add into a cleared Z)?
+bool tc_backward_update_splits(const codenet_layer_impl& L, int B);
 // Output deviations of the feedforward nodes whose own input copy the plan hits, into L.ws.dY (zeroed first).
 cudaError_t launch_input_faults(const codenet_layer_impl& L, int B, cudaStream_t st);
 // Injection, detection, location, decoding plan and the final sums over codewords.

@@ -93,6 +93,7 @@ struct EmitOperands {
   float* xT; float* dT;
   __nv_bfloat16* xb; __nv_bfloat16* dpair;
   size_t dcount;
+  float4* clear; size_t clear_n16;   // a buffer to fill with zeros on the way (16-byte units), or NULL
 };
 
 __global__ void __launch_bounds__(128)
@@ -101,6 +102,9 @@ encode_vectors_kernel(Geom g, const float* __restrict__ X, const float* __restri
                       float* __restrict__ xsum, int vec_ok, LossFuse lf, EmitOperands em, SmallDev sf) {
   __shared__ float red[4];
   __shared__ int s_last, s_enc_hit;
+  if (em.clear != nullptr)
+    for (size_t c = blockIdx.x * (size_t)blockDim.x + threadIdx.x; c < em.clear_n16; c += (size_t)gridDim.x * blockDim.x)
+      em.clear[c] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
   const int nxseg = X ? g.Nn * g.nsc * B : 0;
   int seg = blockIdx.x;
   float part = 0.0f, loss_part = 0.0f;
@@ -544,7 +548,8 @@ cudaError_t launch_encode_layer(const Geom& g, const void* W, cudaStream_t st) {
 }
 
 cudaError_t launch_encode_vectors(const codenet_layer_impl& L, const float* X, const float* Delta,
-                                  int B, cudaStream_t st, const LossFuse* fuse, int emit, const SmallDev* small) {
+                                  int B, cudaStream_t st, const LossFuse* fuse, int emit, const SmallDev* small,
+                                  float* clear, size_t clear_floats) {
   const Geom& g = L.g;
   const int nseg = (X ? g.Nn * g.nsc * B : 0) + (Delta ? g.M * g.ns * B : 0);
   if (nseg == 0) return cudaSuccess;
@@ -558,6 +563,11 @@ cudaError_t launch_encode_vectors(const codenet_layer_impl& L, const float* X, c
                       (reinterpret_cast<uintptr_t>(lf.S) & 15u) == 0 && (reinterpret_cast<uintptr_t>(lf.target) & 15u) == 0;
   EmitOperands em;
   em.xT = nullptr; em.dT = nullptr; em.xb = nullptr; em.dpair = nullptr; em.dcount = (size_t)B * g.Mbr;
+  em.clear = nullptr; em.clear_n16 = 0;
+  if (clear != nullptr && (reinterpret_cast<uintptr_t>(clear) & 15u) == 0 && clear_floats % 4 == 0) {
+    em.clear = reinterpret_cast<float4*>(clear); em.clear_n16 = clear_floats / 4;
+    L.z_cleared = 1;
+  }
   L.operands_ready = 0;
   // (the bfloat16 copies move 8 bytes per four entries: padded widths that are multiples of four make them aligned)
   if (emit != 0 && vec_ok && X && Delta && g.ldb % 4 == 0 && g.ld % 4 == 0) {

@@ -399,12 +399,28 @@ cudaError_t launch_tc_forward(const codenet_layer_impl& L, const float* X, int B
   cudaError_t e;
   ProfileScope scope(CODENET_KERNEL_FORWARD, st);
   if (tf32) {
-    constexpr int MT = 2, SPLIT = 1, STAGES = 4;
-    const size_t smem = (size_t)STAGES * (MT * TC_TILE_M + SPLIT * B) * TC_KBYTES + 1024;
-    dim3 grid((g.Mbr + MT * TC_TILE_M - 1) / (MT * TC_TILE_M), g.n);
-    e = cudaFuncSetAttribute(tc_products_kernel<true, MT, SPLIT, STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    tc_products_kernel<true, MT, SPLIT, STAGES, false><<<grid, TC_THREADS, smem, st>>>(mapW, mapX, p);
+    int sms = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    constexpr int SPLIT = 1, STAGES = 4;
+    const long ctas2 = (long)((g.Mbr + 2 * TC_TILE_M - 1) / (2 * TC_TILE_M)) * g.n;
+    if (ctas2 * 4 < (long)sms * 3) {
+      // two row tiles per CTA would leave a quarter of the SMs and more without one (configuration 5: 80 CTAs):
+      // one tile per CTA, two CTAs fit an SM
+      constexpr int MT = 1;
+      const size_t smem = (size_t)STAGES * (MT * TC_TILE_M + SPLIT * B) * TC_KBYTES + 1024;
+      dim3 grid((g.Mbr + MT * TC_TILE_M - 1) / (MT * TC_TILE_M), g.n);
+      e = cudaFuncSetAttribute(tc_products_kernel<true, MT, SPLIT, STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      tc_products_kernel<true, MT, SPLIT, STAGES, false><<<grid, TC_THREADS, smem, st>>>(mapW, mapX, p);
+    } else {
+      constexpr int MT = 2;
+      const size_t smem = (size_t)STAGES * (MT * TC_TILE_M + SPLIT * B) * TC_KBYTES + 1024;
+      dim3 grid((g.Mbr + MT * TC_TILE_M - 1) / (MT * TC_TILE_M), g.n);
+      e = cudaFuncSetAttribute(tc_products_kernel<true, MT, SPLIT, STAGES, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+      if (e != cudaSuccess) return e;
+      tc_products_kernel<true, MT, SPLIT, STAGES, false><<<grid, TC_THREADS, smem, st>>>(mapW, mapX, p);
+    }
   } else {
     // Two or three 128-row tiles per CTA.  The kernel sits at the bandwidth between L2 and the SM (the hi + lo
     // operand tiles of a K step are as many bytes as two weight tiles), so what a K step moves per weight tile
@@ -784,6 +800,8 @@ namespace {
 struct TcFusedParams {
   Geom g;
   int B, n_rt, n_items;   // row tiles per block-row; work items (block-row, column tile)
+  int zsplit;             // an item's row tiles are shared out among this many CTAs (1 or 2); with 2 each adds its part
+                          // of Z into a buffer cleared before the launch (two addends: the sum does not depend on the order)
   float lr;
   float* Z;               // [block-row][block-column][position][b], or NULL
   int* flag;
@@ -861,7 +879,10 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
   const uint32_t tmem_z = tmem + 256;
 
   // item -> (block-row, column tile); tiles of the absent corner (parity row x parity column) are not items
-  auto item_of = [&](int item, int* i_blk, int* ct) {
+  const int n_units = p.n_items * p.zsplit, rt_per = p.n_rt / p.zsplit;
+  auto item_of = [&](int unit, int* i_blk, int* ct, int* rt0) {
+    const int item = unit / p.zsplit;
+    *rt0 = (unit % p.zsplit) * rt_per;
     const int data_items = p.g.m * n_ct;
     if (item < data_items) { *i_blk = item / n_ct; *ct = item % n_ct; }
     else {
@@ -876,11 +897,11 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
     const uint64_t w_pol = l2_evict_first();
     uint32_t wn = 0, dn = 0, xn = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++xn) {
-      int i_blk, ct;
-      item_of(item, &i_blk, &ct);
+    for (int item = blockIdx.x; item < n_units && ok; item += gridDim.x, ++xn) {
+      int i_blk, ct, rt0;
+      item_of(item, &i_blk, &ct, &rt0);
       const bool need_z = i_blk < p.g.m && p.Z != nullptr;
-      for (int rt = 0; rt < p.n_rt && ok; ++rt, ++wn) {
+      for (int rt = rt0; rt < rt0 + rt_per && ok; ++rt, ++wn) {
         const int row0 = i_blk * p.g.b_r + rt * TC_TILE_M;
         const uint32_t s = wn % TCF_WST;
         if (wn >= TCF_WST && !mbar_wait(&w_empty[s], ((wn / TCF_WST) - 1) & 1)) { ok = false; break; }
@@ -907,7 +928,7 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
               tma_load_2d(slot + ch * vchunk, &mapD, row0 + ch * EPC, part * B, &d_full[ds]);
           }
         }
-        if (rt == 0 && ok) {   // x~ of this item's columns, after the first tile so that it never delays it
+        if (rt == rt0 && ok) {   // x~ of this item's columns, after the first tile so that it never delays it
           if (xn >= 1 && !mbar_wait(&x_empty, (xn - 1) & 1)) { ok = false; break; }
           mbar_expect_tx(&x_full, vtile);
           if (TF32) {
@@ -927,18 +948,18 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
     constexpr uint64_t kstep_mn = (uint64_t)(KI * TC_KBYTES) >> 4;   // KI K rows of an MN-major tile
     uint32_t wn = 0, dn = 0, xn = 0, zn = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x, ++xn) {
-      int i_blk, ct;
-      item_of(item, &i_blk, &ct);
+    for (int item = blockIdx.x; item < n_units && ok; item += gridDim.x, ++xn) {
+      int i_blk, ct, rt0;
+      item_of(item, &i_blk, &ct, &rt0);
       const bool need_z = i_blk < p.g.m && p.Z != nullptr;
-      for (int rt = 0; rt < p.n_rt && ok; ++rt, ++wn) {
+      for (int rt = rt0; rt < rt0 + rt_per && ok; ++rt, ++wn) {
         const uint32_t s = wn % TCF_WST, u = wn & 1;
         if (!mbar_wait(&w_full[s], (wn / TCF_WST) & 1)) { ok = false; break; }
         uint32_t ds = dn % TCF_DST;
         if (!mbar_wait(&d_full[ds], (dn / TCF_DST) & 1)) { ok = false; break; }
-        if (rt == 0 && !mbar_wait(&x_full, xn & 1)) { ok = false; break; }
+        if (rt == rt0 && !mbar_wait(&x_full, xn & 1)) { ok = false; break; }
         if (wn >= 2 && !mbar_wait(&acc_empty[u], ((wn >> 1) - 1) & 1)) { ok = false; break; }
-        if (rt == 0 && need_z && zn >= 1 && !mbar_wait(&z_empty, (zn - 1) & 1)) { ok = false; break; }
+        if (rt == rt0 && need_z && zn >= 1 && !mbar_wait(&z_empty, (zn - 1) & 1)) { ok = false; break; }
         tc_fence_after();
         const uint8_t* wt = sW + (size_t)s * TCF_WTILE;
         const uint8_t* dt = sD + (size_t)ds * dslot;
@@ -974,7 +995,7 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
 #pragma unroll
             for (int kk = 0; kk < TC_TILE_M / KI; ++kk) {
               const uint64_t db = smem_desc_k128(dz + (kk / KPC) * vchunk) + (uint64_t)((kk % KPC) * 2);
-              tc_mma<TF32>(tmem_z, da + (uint64_t)kk * kstep_mn, db, idesc_z, (rt > 0 || part > 0 || kk > 0) ? 1u : 0u);
+              tc_mma<TF32>(tmem_z, da + (uint64_t)kk * kstep_mn, db, idesc_z, (rt > rt0 || part > 0 || kk > 0) ? 1u : 0u);
             }
           }
           if (!ok) break;
@@ -996,11 +1017,11 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
     const int row = quad * 32 + lane;             // tile row (update) or tile column (Z) of this thread
     uint32_t wn = 0, zn = 0;
     bool alive = true;
-    for (int item = blockIdx.x; item < p.n_items && alive; item += gridDim.x) {
-      int i_blk, ct;
-      item_of(item, &i_blk, &ct);
+    for (int item = blockIdx.x; item < n_units && alive; item += gridDim.x) {
+      int i_blk, ct, rt0;
+      item_of(item, &i_blk, &ct, &rt0);
       const bool need_z = i_blk < p.g.m && p.Z != nullptr;
-      for (int rt = 0; rt < p.n_rt; ++rt, ++wn) {
+      for (int rt = rt0; rt < rt0 + rt_per; ++rt, ++wn) {
         const uint32_t s = wn % TCF_WST, u = wn & 1;
         if (!mbar_wait(&acc_full[u], (wn >> 1) & 1) || !mbar_wait(&w_read[s], (wn / TCF_WST) & 1)) { alive = false; break; }
         tc_fence_after();
@@ -1056,12 +1077,18 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
         for (int b0 = half * (B / 2); b0 < (half + 1) * (B / 2); b0 += 32) {
           uint32_t r[32];
           tmem_ld32(tmem_z + ((uint32_t)(quad * 32) << 16) + (uint32_t)b0, r);
-          if (valid) {
+          if (valid && p.zsplit == 1) {
             float4* dst = reinterpret_cast<float4*>(zrow + b0);
 #pragma unroll
             for (int q = 0; q < 8; ++q)
               dst[q] = make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]),
                                    __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+          } else if (valid) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                           :: "l"(zrow + b0 + 4 * q), "f"(__uint_as_float(r[4 * q])), "f"(__uint_as_float(r[4 * q + 1])),
+                              "f"(__uint_as_float(r[4 * q + 2])), "f"(__uint_as_float(r[4 * q + 3])) : "memory");
           }
         }
         tc_fence_before();
@@ -1076,10 +1103,10 @@ tc_backward_update_kernel(const __grid_constant__ CUtensorMap mapW, const __grid
     const uint64_t w_pol = l2_evict_first();
     uint32_t wn = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < p.n_items && ok; item += gridDim.x) {
-      int i_blk, ct;
-      item_of(item, &i_blk, &ct);
-      for (int rt = 0; rt < p.n_rt; ++rt, ++wn) {
+    for (int item = blockIdx.x; item < n_units && ok; item += gridDim.x) {
+      int i_blk, ct, rt0;
+      item_of(item, &i_blk, &ct, &rt0);
+      for (int rt = rt0; rt < rt0 + rt_per; ++rt, ++wn) {
         const uint32_t s = wn % TCF_WST;
         if (!mbar_wait(&w_done[s], (wn / TCF_WST) & 1)) { ok = false; break; }
         const int row0 = i_blk * p.g.b_r + rt * TC_TILE_M;
@@ -1170,6 +1197,22 @@ bool tc_backward_update_supported(const Geom& g, int math, int B) {
   return B % 64 == 0 && B <= 128 && tcf_smem_bytes(tf32, B) <= 227 * 1024;
 }
 
+// One CTA per SM walks whole items; when the items do not fill the last round of CTAs (configuration 5: 192 items on
+// 148 SMs, two rounds for 1.3 rounds' worth of work) halves of items even the rounds out.  Taken only where it saves
+// a fifth of the rounds: the halves add into Z, which costs a clearing pass over it.
+bool tc_backward_update_splits(const codenet_layer_impl& L, int B) {
+  const Geom& g = L.g;
+  if (!tc_backward_update_supported(g, L.desc.math, B)) return false;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int n_rt = g.b_r / TC_TILE_M;
+  const long n_items = (long)g.m * (g.ld / TC_TILE_M) + (long)g.r_row * g.n * (g.ldb / TC_TILE_M);
+  if (n_rt % 2 != 0) return false;
+  const long whole = (n_items + sms - 1) / sms * 2, halves = (2 * n_items + sms - 1) / sms;
+  return halves * 5 <= whole * 4;
+}
+
 cudaError_t launch_tc_backward_update(const codenet_layer_impl& L, int B, float lr, float* Z, cudaStream_t st) {
   const Geom& g = L.g;
   const bool tf32 = g.dtype == CODENET_F32;
@@ -1228,7 +1271,15 @@ cudaError_t launch_tc_backward_update(const codenet_layer_impl& L, int B, float 
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int grid = p.n_items < sms ? p.n_items : sms;
+  p.zsplit = (Z != nullptr && tc_backward_update_splits(L, B)) ? 2 : 1;
+  const bool cleared = L.z_cleared != 0;   // (by the vector-encoding kernel, on its way)
+  L.z_cleared = 0;
+  if (p.zsplit == 2 && !cleared) {
+    e = cudaMemsetAsync(Z, 0, (size_t)g.m * g.Nn * g.b_c * B * sizeof(float), st);
+    if (e != cudaSuccess) return e;
+  }
+  const int units = p.n_items * p.zsplit;
+  const int grid = units < sms ? units : sms;
   ProfileScope scope(CODENET_KERNEL_BACKWARD_UPDATE, st);
   if (tf32) tc_backward_update_kernel<true><<<grid, TCF_THREADS, smem, st>>>(mapW, mapD, mapX, mapDu, p);
   else tc_backward_update_kernel<false><<<grid, TCF_THREADS, smem, st>>>(mapW, mapD, mapX, mapDu, p);
