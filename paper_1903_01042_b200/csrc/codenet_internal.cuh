@@ -58,6 +58,8 @@ struct CheckStats {
   unsigned syn[CODENET_MAX_NODES];                        // [codeword] max |syndrome|
   unsigned resid[CODENET_MAX_NODES];                      // [codeword] max residual of the decoding plan
   unsigned need_fix, done_d;
+  unsigned fix_go;   // written by the CTA of the last codeword to decide: 1 = no codeword needs work, 2 = some do
+  unsigned pad_;
 };
 
 // Per-codeword decision and erasure-decoding plan.

@@ -442,6 +442,10 @@ __device__ __forceinline__ void checksum_dot(const float* a, const float* w, int
   }
 }
 
+template <bool SPARE>
+__device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, const float* sP, const unsigned long long* s_inj,
+                                         const unsigned bid, const unsigned gdim);
+
 // PAIR: the body runs as one part of a paired launch (p.pair says which); bid / gdim are the CTA's index and the
 // number of CTAs within its part.  Both parts pass the same two grid barriers.
 template <bool BIG, bool PAIR>
@@ -1248,7 +1252,7 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
         atomicMax(reinterpret_cast<unsigned*>(&r->max_margin_clean), __float_as_uint(cw_max_clean));
       }
       s_last = 0;
-      if (p.inline_fix) {
+      if (p.inline_fix || p.tail_fix) {
         // only the in-kernel fix needs to know which CTA comes last; the same counter carries, above bit 16,
         // how many codewords need work, so the last CTA learns both from one atomic
         __threadfence();
@@ -1260,7 +1264,13 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
       }
     }
     __syncthreads();
-    if (s_last) {  // the CTA of the last codeword to decide finishes the job
+    if (s_last && p.tail_fix) {
+      // every plan is written: tell the waiting grid whether there is anything to do
+      if (tid == 0) {
+        __threadfence();
+        atomicExch(&p.st->fix_go, (unsigned)s_last);
+      }
+    } else if (s_last) {  // the CTA of the last codeword to decide finishes the job
       __threadfence();
       const bool fix_here = p.inline_fix && p.out != nullptr && s_last == 2;
       if (fix_here) {
@@ -1300,6 +1310,25 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
       }
     }
   }
+  if (BIG && p.tail_fix) {
+    // Large batches: the whole (co-resident) grid waits for the word the last deciding CTA writes -- a bounded
+    // wait, about a microsecond in the usual case where nothing was detected -- and does the fix kernel's work
+    // together when some codeword needs it: no second launch behind every check.
+    __shared__ unsigned s_go;
+    if (tid == 0) {
+      unsigned v = 0u;
+      for (unsigned spin = 0; spin < (1u << 22); ++spin) {
+        v = *reinterpret_cast<volatile unsigned*>(&p.st->fix_go);
+        if (v != 0u) break;
+        __nanosleep(64);
+      }
+      if (v == 0u) atomicExch(const_cast<int*>(p.tc_flag), 1);   // gave up: reported as TIMEOUT by the next check
+      __threadfence();
+      s_go = v;
+    }
+    __syncthreads();
+    if (s_go == 2u) fix_body<false>(p, q, sP, s_inj, bid, gdim);
+  }
   // every CTA read the counter before the first grid barrier
   if (p.bump != nullptr && bid == 0 && tid == 0) *p.bump += 1u;
 }
@@ -1328,23 +1357,18 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_pair_kernel(const __grid_
 // SPARE: some plan may have a spare parity to be verified on (two and more parities in the phase's code);
 // that pass needs a grid barrier, so only this instantiation is a cooperative launch.
 template <bool SPARE>
-__global__ void __launch_bounds__(CK_THREADS) fix_kernel(CheckParams p) {
-  p.st = p.st_base + ((__ldcg(p.parity) & 1) ^ 1);   // the buffer the check kernel before this one worked in
-  if (p.st->need_fix == 0u) return;  // the usual case: every codeword passed its checks
+__device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, const float* sP, const unsigned long long* s_inj,
+                                         const unsigned bid, const unsigned gdim) {
   const Geom& g = p.g;
   const bool fwd = p.phase == CODENET_PHASE_FWD;
-  const PhaseGeom q = phase_geom(g, p.phase, p.B);
   const int B = p.B;
   const int tid = threadIdx.x;
-  __shared__ float sP[MAXN * MAXR];
-  __shared__ unsigned long long s_inj[MAXN];
   __shared__ unsigned s_res[MAXN];
   __shared__ unsigned s_final[MAXN];
-  for (int t = tid; t < q.kd * q.r; t += CK_THREADS) sP[t] = q.P[t];
   for (int t = tid; t < MAXN; t += CK_THREADS) s_res[t] = 0u;
-  build_hit_masks(p, q, s_inj);
-  const size_t gstride = (size_t)gridDim.x * CK_THREADS;
-  const size_t g0 = blockIdx.x * (size_t)CK_THREADS + tid;
+  __syncthreads();
+  const size_t gstride = (size_t)gdim * CK_THREADS;
+  const size_t g0 = bid * (size_t)CK_THREADS + tid;
 
   // phase V: residual of every decoding plan on its spare parities
   if (SPARE) {
@@ -1436,10 +1460,22 @@ __global__ void __launch_bounds__(CK_THREADS) fix_kernel(CheckParams p) {
       }
     }
   }
-  if (p.rep && blockIdx.x == 0) {
+  if (p.rep && bid == 0) {
     __shared__ float s_a[MAXN], s_b[MAXN];
     write_report(p, q.n_cw, s_final, s_a, s_b);
   }
+}
+
+template <bool SPARE>
+__global__ void __launch_bounds__(CK_THREADS) fix_kernel(CheckParams p) {
+  p.st = p.st_base + ((__ldcg(p.parity) & 1) ^ 1);   // the buffer the check kernel before this one worked in
+  if (p.st->need_fix == 0u) return;  // the usual case: every codeword passed its checks
+  const PhaseGeom q = phase_geom(p.g, p.phase, p.B);
+  __shared__ float sP[MAXN * MAXR];
+  __shared__ unsigned long long s_inj[MAXN];
+  for (int t = threadIdx.x; t < q.kd * q.r; t += CK_THREADS) sP[t] = q.P[t];
+  build_hit_masks(p, q, s_inj);
+  fix_body<SPARE>(p, q, sP, s_inj, blockIdx.x, gridDim.x);
 }
 
 // Soft errors in a node's own copy of its input sub-vector (the copy the activation / post-multiplication step
@@ -1554,7 +1590,7 @@ void fill_check_params(const codenet_layer_impl& L, int phase, const float* src,
   p.out_act = phase == CODENET_PHASE_FWD ? L.out_act : CODENET_ACT_IDENTITY;
   p.out_mask = phase == CODENET_PHASE_BWD ? L.out_mask : nullptr;
   if (phase == CODENET_PHASE_FWD) L.out_act = CODENET_ACT_IDENTITY; else L.out_mask = nullptr;
-  p.lazy = 0; p.inline_fix = 0; p.bump = nullptr;
+  p.lazy = 0; p.inline_fix = 0; p.tail_fix = 0; p.bump = nullptr;
   p.it_add = 0u; p.pair = 0; p.pair_sums = nullptr;
   p.commit_S = nullptr; p.commit_S_to = nullptr; p.commit_n = 0; p.commit_rep = nullptr; p.commit_rep_to = nullptr;
   p.loss_partials = nullptr; p.loss_n = 0; p.loss_out = nullptr;
@@ -1663,10 +1699,12 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
   p.lazy = big ? 1 : 0;
   p.bump = nullptr;
   p.inline_fix = (!big && B <= 8 && (fwd ? g.r_row : g.r_col) <= 1 && !commit && out != nullptr) ? 1 : 0;
+  // large batches with at most one parity: the grid waits for the last decision and fixes together (check_body)
+  p.tail_fix = (big && (fwd ? g.r_row : g.r_col) <= 1 && !commit && out != nullptr) ? 1 : 0;
   const size_t cap = big ? (size_t)g_coop_blocks_check_max : (size_t)g_coop_blocks_check;
   int grid_c = (int)(want < cap ? want : cap);
   int grid_f = (int)(by_el < (size_t)g_coop_blocks_fix ? (by_el < 1 ? 1 : by_el) : (size_t)g_coop_blocks_fix);
-  if (L.bump_after != nullptr && !fwd && p.inline_fix) {   // (with a fix kernel behind, the counter is still read)
+  if (L.bump_after != nullptr && !fwd && (p.inline_fix || p.tail_fix)) {   // (with a fix kernel behind, the counter is still read)
     p.bump = L.bump_after;
     L.bump_done = true;
   }
@@ -1676,7 +1714,7 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
                                   dim3(grid_c), dim3(CK_THREADS), args, 0, st);
   if (e != cudaSuccess) return e;
   count_launch();
-  if (p.inline_fix) return cudaSuccess;   // the check kernel's last CTA has done what the fix kernel would do
+  if (p.inline_fix || p.tail_fix) return cudaSuccess;   // the check kernel has done what the fix kernel would do
   if ((fwd ? g.r_row : g.r_col) >= 2) {
     e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(fix_kernel<true>), dim3(grid_f), dim3(CK_THREADS), args, 0, st);
   } else {
