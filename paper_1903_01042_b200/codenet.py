@@ -372,12 +372,12 @@ def net_capture_step(net, X_dev, target_dev, lr, faults=None, reps_dev=None, los
 def net_capture_steps(net, X_devs, target_devs, lr, faults=None, reps_dev=None, reps_stride=0, loss_dev=None,
                       loss_stride=0, X_next_dev=None):
     """codenet_net_capture_steps: record len(X_devs) consecutive steps into one CUDA graph; returns its id."""
-    B = X_devs[0].shape[0]
+    B = X_devs[0].shape[0] if len(X_devs) else 0
     for x in X_devs:
         _dev_f32(x, (B, net.layers[0].n_in))
     n = len(X_devs)
-    xs = (C.c_void_p * n)(*[_ptr(x) for x in X_devs])
-    ts = (C.c_void_p * n)(*[_ptr(t) for t in target_devs])
+    xs = (C.c_void_p * max(n, 1))(*[_ptr(x) for x in X_devs])
+    ts = (C.c_void_p * max(n, 1))(*[_ptr(t) for t in target_devs])
     farr = None
     if faults is not None:
         farr = (Fault * len(net.layers))(*faults)

@@ -473,6 +473,23 @@ def test_bad_arguments(cn):
         cn.forward(lay, torch.zeros((3, 8), device="cuda"))  # batch above batch_max
     with pytest.raises(cn.CodenetError):
         cn.get_block(lay, 2, 2)                              # corner: no node
+    x = torch.zeros((1, 8), device="cuda")
+    d = torch.zeros((1, 8), device="cuda")
+    lib = cn.lib()
+    # the combined call needs the next input and a place for its sums
+    assert lib.codenet_backward_update_forward_next(lay.h, d.data_ptr(), x.data_ptr(), 1, 0.01, None, x.data_ptr(), None,
+                                                    None, None, x.data_ptr(), None, None) != 0
+    assert lib.codenet_backward_update_forward_next(lay.h, d.data_ptr(), x.data_ptr(), 1, 0.01, None, x.data_ptr(), None,
+                                                    x.data_ptr(), None, None, None, None) != 0
+    net = cn.net_create([lay], activation=0, loss=0)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        with pytest.raises(cn.CodenetError):
+            cn.net_capture_steps(net, [], [], 0.01)          # no step to record
+    gid = __import__("ctypes").c_int(-1)
+    assert lib.codenet_net_capture_steps(net.h, 1, None, None, 1, 0.01, None, None, 0, None, 0, None, side.cuda_stream,
+                                         __import__("ctypes").byref(gid)) != 0      # no input list
+    assert lib.codenet_net_set_iteration_counter(None, None) != 0
 
 
 # ---------------------------------------------------------------------------------------------
