@@ -1310,10 +1310,11 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
       }
     }
   }
-  if (BIG && p.tail_fix) {
-    // Large batches: the whole (co-resident) grid waits for the word the last deciding CTA writes -- a bounded
-    // wait, about a microsecond in the usual case where nothing was detected -- and does the fix kernel's work
-    // together when some codeword needs it: no second launch behind every check.
+  if (!PAIR && p.tail_fix) {
+    // The whole (co-resident) grid waits for the word the last deciding CTA writes -- a bounded wait, about a
+    // microsecond in the usual case where nothing was detected -- and does the fix kernel's work together when
+    // some codeword needs it (with two and more parities that includes the pass over the spare parities and its
+    // grid barrier, which every CTA then takes): no second launch behind every check.
     __shared__ unsigned s_go;
     if (tid == 0) {
       unsigned v = 0u;
@@ -1327,7 +1328,10 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
       s_go = v;
     }
     __syncthreads();
-    if (s_go == 2u) fix_body<false>(p, q, sP, s_inj, bid, gdim);
+    if (s_go == 2u) {
+      if (q.r >= 2) fix_body<true>(p, q, sP, s_inj, bid, gdim);
+      else fix_body<false>(p, q, sP, s_inj, bid, gdim);
+    }
   }
   // every CTA read the counter before the first grid barrier
   if (p.bump != nullptr && bid == 0 && tid == 0) *p.bump += 1u;
@@ -1699,8 +1703,8 @@ cudaError_t launch_check(const codenet_layer_impl& L, int phase, const float* sr
   p.lazy = big ? 1 : 0;
   p.bump = nullptr;
   p.inline_fix = (!big && B <= 8 && (fwd ? g.r_row : g.r_col) <= 1 && !commit && out != nullptr) ? 1 : 0;
-  // large batches with at most one parity: the grid waits for the last decision and fixes together (check_body)
-  p.tail_fix = (big && (fwd ? g.r_row : g.r_col) <= 1 && !commit && out != nullptr) ? 1 : 0;
+  // large batches, or two and more parities: the grid waits for the last decision and fixes together (check_body)
+  p.tail_fix = ((big || (fwd ? g.r_row : g.r_col) >= 2) && !p.inline_fix && !commit && out != nullptr) ? 1 : 0;
   const size_t cap = big ? (size_t)g_coop_blocks_check_max : (size_t)g_coop_blocks_check;
   int grid_c = (int)(want < cap ? want : cap);
   int grid_f = (int)(by_el < (size_t)g_coop_blocks_fix ? (by_el < 1 ? 1 : by_el) : (size_t)g_coop_blocks_fix);
