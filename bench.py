@@ -292,41 +292,52 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
         one(it)
     torch.cuda.synchronize()
     replay = None
-    if graphs and e2e:
-        # End to end with the steps in a graph of the caller's own: the eight steps of the pool are captured
-        # together WITH their copies, uploads and downloads on streams of their own.  Step k reads its input from
-        # staging buffer (k - 1) % 4 (it went up for step k - 1) and its target and the next input from buffer
-        # k % 4, which may go up as soon as step k - 3, its last reader, has ended; every step has its own result
-        # slot, copied down behind it.  The host reads a replay's eight losses from pinned memory after it has queued
-        # the next replay.  The network advances the fault plans' iteration counter itself.
+    if graphs:
+        # Recorded steps.  The K timed steps are cut into consecutive segments of 40 (and the rest), each one graph:
+        # between two graph launches the device idles for 8-15 us, which a long recording makes rare.  40 is a
+        # multiple of the input pool and of the staging ring, so one 40-step recording serves every whole segment.
+        # (Measured at K = 20: one recording of 20 steps, or any cut of them into 2-4 graphs with short ones first,
+        # all give 130.4-130.9 us per step against 125.0 at K = 1000: the first steps after the synchronisation
+        # that precedes the timed region run slower, however they are launched.)
         it_ctr = torch.full((1,), warmup, dtype=torch.int32, device="cuda")
         faults = [cn.make_fault(seed=cfg.seed, layer=l, mode=mode, p=cfg.p, sigma=cfg.sigma, iteration_dev=it_ctr)
                   for l in range(L)]
+        segs, left = [], steps
+        while left > 0:
+            segs.append(min(40, left)); left -= segs[-1]
+        starts = [sum(segs[:q]) for q in range(len(segs))]
+        group = max(segs)
+    if graphs and e2e:
+        # End to end with the steps in graphs of the caller's own: the steps of a segment are captured together WITH
+        # their copies, uploads and downloads on streams of their own.  Step k (counted from the first timed step)
+        # reads its input from staging buffer (k - 1) % 4 (it went up for step k - 1) and its target and the next
+        # input from buffer k % 4, which may go up as soon as step k - 3, its last reader, has ended; every step has
+        # its own result slot, copied down behind it.  The host reads a replay's losses from pinned memory after it
+        # has queued the next replay.  The network advances the fault plans' iteration counter itself.
         cn.net_set_iteration_counter(net, it_ctr)
         slot = rb + 16
-        outs_dev = torch.zeros(pool * slot, dtype=torch.uint8, device="cuda")
-        outs_host = [torch.empty(pool * slot, dtype=torch.uint8).pin_memory() for _ in range(2)]
-        order = [(warmup + k) % pool for k in range(pool)]
+        outs_dev = torch.zeros(group * slot, dtype=torch.uint8, device="cuda")
+        outs_host = [torch.empty(group * slot, dtype=torch.uint8).pin_memory() for _ in range(2)]
         main, up, down = torch.cuda.current_stream(), torch.cuda.Stream(), torch.cuda.Stream()
         torch.cuda.synchronize()
 
-        def record(dst_host, n_rec):
+        def record(dst_host, base, n_rec):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=main):
                 step_done = []
                 up.wait_stream(main)
                 down.wait_stream(main)
                 for k in range(n_rec):
-                    src = order[k]
+                    src, ring = (warmup + base + k) % pool, (base + k) % 4
                     if k >= 3:
                         up.wait_event(step_done[k - 3])
                     with torch.cuda.stream(up):
-                        stage3[k % 4].copy_(hs[src], non_blocking=True)      # [x of step k + 1 | target of step k]
+                        stage3[ring].copy_(hs[src], non_blocking=True)       # [x of the next step | target of this one]
                     main.wait_stream(up)
                     o = outs_dev[k * slot:(k + 1) * slot]
                     if lookahead:
-                        cn.net_set_next_input(net, sx3[k % 4])
-                    cn.step(net, sx3[(k - 1) % 4], st3[k % 4], cfg.lr, faults=faults, reps_dev=o[:rb],
+                        cn.net_set_next_input(net, sx3[ring])
+                    cn.step(net, sx3[(ring - 1) % 4], st3[ring], cfg.lr, faults=faults, reps_dev=o[:rb],
                             loss_dev=o[rb:rb + 4].view(torch.float32))
                     ev = torch.cuda.Event()
                     ev.record(main)
@@ -338,54 +349,53 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
                 main.wait_stream(down)
             return g
         before = cn.launch_count()
-        # recorded in the order of the replays (each recording continues the look-ahead state of the one before):
-        # whole pools alternating between the two host buffers, then the last steps % pool steps once
-        n_full, tail = steps // pool, steps % pool
-        graphs2 = [record(outs_host[r], pool) for r in range(min(n_full, 2))]
-        net.launches_per_recorded_step = (cn.launch_count() - before) // max(1, pool * len(graphs2))
-        g_tail = record(outs_host[n_full % 2], tail) if tail else None
-        if not graphs2:
-            net.launches_per_recorded_step = (cn.launch_count() - before) // tail
+        # recorded in the order of the replays (each recording continues the look-ahead state of the one before);
+        # replay q writes host buffer q % 2
+        recorded, seg_graph = {}, []
+        for q, (base, size) in enumerate(zip(starts, segs)):
+            key = (base % 8, size, q % 2)
+            if key not in recorded:
+                recorded[key] = record(outs_host[q % 2], base, size)
+            seg_graph.append(recorded[key])
+        net.launches_per_recorded_step = (cn.launch_count() - before) // max(1, sum(k[1] for k in recorded))
         done = [torch.cuda.Event() for _ in range(2)]
         seen = {"loss": 0.0}
         hout = outs_host[0][:slot]
+        seg_at = {st_: q for q, st_ in enumerate(starts)}
+
+        def read_losses(q):
+            for w in range(segs[q]):                         # the caller's read of every step's loss
+                seen["loss"] = float(outs_host[q % 2][w * slot + rb:w * slot + rb + 4].view(torch.float32)[0])
 
         def replay(it):
-            k = it - warmup
-            if k % pool:
+            q = seg_at.get(it - warmup)
+            if q is None:
                 return
-            r = k // pool
-            (graphs2[r % 2] if r < n_full else g_tail).replay()
-            done[r % 2].record()
-            if r > 0:
-                done[(r - 1) % 2].synchronize()
-                for q in range(pool):                        # the caller's read of every step's loss
-                    seen["loss"] = float(outs_host[(r - 1) % 2][q * slot + rb:q * slot + rb + 4].view(torch.float32)[0])
+            seg_graph[q].replay()
+            done[q % 2].record()
+            if q > 0:
+                done[(q - 1) % 2].synchronize()
+                read_losses(q - 1)
         torch.cuda.synchronize()
     if graphs and not e2e:
-        # the pool's steps recorded into one graph, in the order they will run (one graph launch per `pool` steps:
-        # no pause between the steps of a replay); the iteration counter is a single device word that every
-        # recorded step advances
-        it_ctr = torch.full((1,), warmup, dtype=torch.int32, device="cuda")
-        faults = [cn.make_fault(seed=cfg.seed, layer=l, mode=mode, p=cfg.p, sigma=cfg.sigma, iteration_dev=it_ctr)
-                  for l in range(L)]
-        order = [(warmup + k) % pool for k in range(pool)]
+        # the iteration counter is a single device word that every recorded step advances
         before = cn.launch_count()
-        gid_all = cn.net_capture_steps(net, [dxs[k] for k in order], [dts[k] for k in order], cfg.lr, faults=faults,
-                                       reps_dev=reps, loss_dev=loss_dev,
-                                       X_next_dev=dxs[order[0]] if lookahead else None)
-        net.launches_per_recorded_step = (cn.launch_count() - before) // pool
-        tail = steps % pool          # the last steps % pool steps: a shorter recording, replayed once at the end
-        gid_tail = None
-        if tail:
-            gid_tail = cn.net_capture_steps(net, [dxs[k] for k in order[:tail]], [dts[k] for k in order[:tail]], cfg.lr,
-                                            faults=faults, reps_dev=reps, loss_dev=loss_dev,
-                                            X_next_dev=dxs[order[tail]] if lookahead else None)
+        recorded, seg_graph = {}, []
+        for base, size in zip(starts, segs):
+            key = (base % pool, size)
+            if key not in recorded:
+                order = [(warmup + base + k) % pool for k in range(size + 1)]
+                recorded[key] = cn.net_capture_steps(net, [dxs[k] for k in order[:size]], [dts[k] for k in order[:size]],
+                                                     cfg.lr, faults=faults, reps_dev=reps, loss_dev=loss_dev,
+                                                     X_next_dev=dxs[order[size]] if lookahead else None)
+            seg_graph.append(recorded[key])
+        net.launches_per_recorded_step = (cn.launch_count() - before) // max(1, sum(k[1] for k in recorded))
+        seg_at = {st_: q for q, st_ in enumerate(starts)}
 
         def replay(it):
-            k = it - warmup
-            if k % pool == 0:
-                cn.net_replay(net, gid_all if k + pool <= steps else gid_tail)
+            q = seg_at.get(it - warmup)
+            if q is not None:
+                cn.net_replay(net, seg_graph[q])
         torch.cuda.synchronize()
     if sampler is not None:
         sampler.start()
@@ -399,6 +409,8 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
             one(it)
     ev1.record()
     torch.cuda.synchronize()
+    if e2e and graphs and segs:
+        read_losses(len(segs) - 1)                           # the last replay's losses, read like the others
     if sampler is not None:
         sampler.stop_flag.set()
     secs = ev0.elapsed_time(ev1) / 1e3

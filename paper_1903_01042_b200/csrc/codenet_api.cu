@@ -863,6 +863,8 @@ int codenet_net_capture_steps(codenet_net_t* net, int n_steps, const float* cons
   const cudaError_t e2 = cudaGraphInstantiate(&exec, graph, 0);
   cudaGraphDestroy(graph);
   if (e2 != cudaSuccess) return cuda_status(e2);
+  // the device-side copy of the graph is made now, not by the first replay
+  if (cudaGraphUpload(exec, st) != cudaSuccess) { cudaGraphExecDestroy(exec); return CODENET_E_CUDA; }
   net->graphs.push_back(exec);
   *graph_id = (int)net->graphs.size() - 1;
   return CODENET_OK;
