@@ -399,6 +399,7 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
         torch.cuda.synchronize()
     if sampler is not None:
         sampler.start()
+    torch.cuda.synchronize()
     launches0 = cn.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
