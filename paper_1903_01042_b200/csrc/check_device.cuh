@@ -299,35 +299,49 @@ __device__ __forceinline__ void syndrome_at(const CwView& yw, const PhaseGeom& q
 // lowest-indexed unlocated parities; par[] receives every parity re-encoded from the result.
 __device__ __forceinline__ void decode_at(const CwView& yw, const PhaseGeom& q, const float* sP, const CwPlan& pl,
                                           size_t e, float (&fix)[MAXR], double (&par)[MAXR]) {
+  // the plan's fields once, into registers (the plan sits in global memory and is the same for every element)
+  const unsigned long long F = pl.F;
+  const int nfd = pl.nfd;
+  int qa[MAXR], fda[MAXR];
+#pragma unroll
+  for (int a = 0; a < MAXR; ++a) { qa[a] = a < nfd ? pl.q[a] : 0; fda[a] = a < nfd ? pl.fd[a] : 0; }
   double rhs[MAXR];
 #pragma unroll
-  for (int a = 0; a < MAXR; ++a) rhs[a] = a < pl.nfd ? (double)yw.at(q, q.kd + pl.q[a], e) : 0.0;
+  for (int a = 0; a < MAXR; ++a) rhs[a] = a < nfd ? (double)yw.at(q, q.kd + qa[a], e) : 0.0;
 #pragma unroll
   for (int t = 0; t < MAXR; ++t) par[t] = 0.0;
-  for (int k = 0; k < q.kd; ++k) {
-    if ((pl.F >> k) & 1ull) continue;
-    const double o = (double)yw.at(q, k, e);
+  // node outputs eight at a time (independent loads, in flight together), used in node order
+  for (int k0 = 0; k0 < q.kd; k0 += 8) {
+    float o8[8];
 #pragma unroll
-    for (int a = 0; a < MAXR; ++a)
-      if (a < pl.nfd) rhs[a] -= (double)sP[k * q.r + pl.q[a]] * o;
+    for (int u = 0; u < 8; ++u) o8[u] = yw.at(q, min(k0 + u, q.kd - 1), e);
 #pragma unroll
-    for (int t = 0; t < MAXR; ++t)
-      if (t < q.r) par[t] += (double)sP[k * q.r + t] * o;
+    for (int u = 0; u < 8; ++u) {
+      const int k = k0 + u;
+      if (k >= q.kd || ((F >> k) & 1ull)) continue;
+      const double o = (double)o8[u];
+#pragma unroll
+      for (int a = 0; a < MAXR; ++a)
+        if (a < nfd) rhs[a] -= (double)sP[k * q.r + qa[a]] * o;
+#pragma unroll
+      for (int t = 0; t < MAXR; ++t)
+        if (t < q.r) par[t] += (double)sP[k * q.r + t] * o;
+    }
   }
 #pragma unroll
   for (int a = 0; a < MAXR; ++a) {
     double acc = 0.0;
 #pragma unroll
     for (int b = 0; b < MAXR; ++b)
-      if (a < pl.nfd && b < pl.nfd) acc += pl.ainv[a * pl.nfd + b] * rhs[b];
+      if (a < nfd && b < nfd) acc += pl.ainv[a * nfd + b] * rhs[b];
     fix[a] = (float)acc;
   }
 #pragma unroll
   for (int a = 0; a < MAXR; ++a)
-    if (a < pl.nfd) {
+    if (a < nfd) {
 #pragma unroll
       for (int t = 0; t < MAXR; ++t)
-        if (t < q.r) par[t] += (double)sP[pl.fd[a] * q.r + t] * (double)fix[a];
+        if (t < q.r) par[t] += (double)sP[fda[a] * q.r + t] * (double)fix[a];
     }
 }
 
@@ -414,5 +428,31 @@ __device__ __forceinline__ float final_value(const CheckParams& p, const PhaseGe
   // uncorrectable: the fault-free recomputation, when there is one
   if (p.have_clean && ((s_inj[cw] >> node) & 1ull)) return clean_value(p, q, cw, node, e);
   return yw.at(q, node, e);
+}
+
+// Sum over the codewords of one output (data node `node`, element e) with final values, in codeword order.  The values
+// of the codewords whose plan does not touch the node (the many) are plain loads, taken eight at a time so that they
+// are in flight together; s_touch[c] holds the nodes codeword c's final plan replaces (decoded or fault-free).
+__device__ __forceinline__ float sum_final_values(const CheckParams& p, const PhaseGeom& q, const float* sP,
+                                                  const unsigned long long* s_inj, const unsigned* s_final,
+                                                  const unsigned long long* s_touch, int node, size_t e) {
+  float acc = 0.0f;
+  for (int c0 = 0; c0 < q.n_cw; c0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int c = min(c0 + u, q.n_cw - 1);
+      v[u] = cw_view(p, q, s_inj, c).at(q, node, e);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int c = c0 + u;
+      if (c < q.n_cw) {
+        if ((s_touch[c] >> node) & 1ull) v[u] = final_value(p, q, sP, s_inj, s_final, c, node, e);
+        acc += v[u];
+      }
+    }
+  }
+  return acc;
 }
 

@@ -1278,10 +1278,12 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
         // are final: the sums of the data nodes they touch are recomputed here, with corrected or
         // fault-free values, in the arithmetic of the fix kernel.
         __shared__ unsigned s_final[MAXN];
-        __shared__ unsigned long long s_nodes;
+        __shared__ unsigned long long s_nodes, s_touch[MAXN];
         if (tid == 0) s_nodes = 0ull;
-        for (int c = tid; c < MAXN; c += CK_THREADS)
+        for (int c = tid; c < MAXN; c += CK_THREADS) {
           s_final[c] = c < q.n_cw ? (unsigned)reinterpret_cast<const volatile CwPlan*>(p.plan)[c].state : 0u;
+          s_touch[c] = 0ull;
+        }
         __syncthreads();
         if (tid < q.n_cw) {
           const volatile CwPlan& pl = p.plan[tid];
@@ -1289,6 +1291,7 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
           unsigned long long mask = 0ull;
           if (s_final[tid] == 1u) mask = pl.F & data;
           else if (s_final[tid] == 3u && p.have_clean) mask = s_inj[tid] & data;
+          s_touch[tid] = mask;
           if (mask) atomicOr(&s_nodes, mask);
         }
         __syncthreads();
@@ -1300,8 +1303,7 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
             const int pos = idx / B, b = idx % B;
             const int gidx = node * q.len + pos;
             if (gidx >= nout) continue;
-            float acc = 0.0f;
-            for (int c = 0; c < q.n_cw; ++c) acc += final_value(p, q, sP, s_inj, s_final, c, node, (size_t)pos * B + b);
+            const float acc = sum_final_values(p, q, sP, s_inj, s_final, s_touch, node, (size_t)pos * B + b);
             const size_t oi = (size_t)b * nout + gidx;
             p.out[oi] = finish_out(p, acc, oi);
           }
@@ -1414,14 +1416,16 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
   // plan touches change (a located parity output, or a failed codeword without a fault-free copy, leaves
   // every sum as the check kernel wrote it), so only their outputs are recomputed.
   if (p.out) {
-    __shared__ unsigned long long s_nodes;
+    __shared__ unsigned long long s_nodes, s_touch[MAXN];
     if (tid == 0) s_nodes = 0ull;
+    for (int c = tid; c < MAXN; c += CK_THREADS) s_touch[c] = 0ull;
     __syncthreads();
     if (tid < q.n_cw) {
       const unsigned long long data = q.kd >= 64 ? ~0ull : ((1ull << q.kd) - 1ull);
       unsigned long long mask = 0ull;
       if (s_final[tid] == 1u) mask = p.plan[tid].F & data;
       else if (s_final[tid] == 3u && p.have_clean) mask = s_inj[tid] & data;
+      s_touch[tid] = mask;
       if (mask) atomicOr(&s_nodes, mask);
     }
     __syncthreads();
@@ -1434,8 +1438,7 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
         const int b = (int)(idx % B), pos = (int)(idx / B);
         const int gidx = node * q.len + pos;
         if (gidx >= nout) continue;
-        float acc = 0.0f;
-        for (int cw = 0; cw < q.n_cw; ++cw) acc += final_value(p, q, sP, s_inj, s_final, cw, node, idx);
+        const float acc = sum_final_values(p, q, sP, s_inj, s_final, s_touch, node, idx);
         p.out[(size_t)b * nout + gidx] = finish_out(p, acc, (size_t)b * nout + gidx);
       }
     }
