@@ -1264,59 +1264,24 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
       }
     }
     __syncthreads();
-    if (s_last && p.tail_fix) {
-      // every plan is written: tell the waiting grid whether there is anything to do
+    if (s_last) {
+      // every plan is written: tell the waiting CTAs whether there is anything to do
       if (tid == 0) {
         __threadfence();
         atomicExch(&p.st->fix_go, (unsigned)s_last);
       }
-    } else if (s_last) {  // the CTA of the last codeword to decide finishes the job
-      __threadfence();
-      const bool fix_here = p.inline_fix && p.out != nullptr && s_last == 2;
-      if (fix_here) {
-        // With at most one parity a decoding plan has no spare parity to be verified against, so the plans
-        // are final: the sums of the data nodes they touch are recomputed here, with corrected or
-        // fault-free values, in the arithmetic of the fix kernel.
-        __shared__ unsigned s_final[MAXN];
-        __shared__ unsigned long long s_nodes, s_touch[MAXN];
-        if (tid == 0) s_nodes = 0ull;
-        for (int c = tid; c < MAXN; c += CK_THREADS) {
-          s_final[c] = c < q.n_cw ? (unsigned)reinterpret_cast<const volatile CwPlan*>(p.plan)[c].state : 0u;
-          s_touch[c] = 0ull;
-        }
-        __syncthreads();
-        if (tid < q.n_cw) {
-          const volatile CwPlan& pl = p.plan[tid];
-          const unsigned long long data = q.kd >= 64 ? ~0ull : ((1ull << q.kd) - 1ull);
-          unsigned long long mask = 0ull;
-          if (s_final[tid] == 1u) mask = pl.F & data;
-          else if (s_final[tid] == 3u && p.have_clean) mask = s_inj[tid] & data;
-          s_touch[tid] = mask;
-          if (mask) atomicOr(&s_nodes, mask);
-        }
-        __syncthreads();
-        const unsigned long long nodes = s_nodes;
-        const int nout = fwd ? g.n_out : g.n_in;
-        for (int node = 0; node < q.kd; ++node) {
-          if (!((nodes >> node) & 1ull)) continue;
-          for (int idx = tid; idx < q.len * B; idx += CK_THREADS) {
-            const int pos = idx / B, b = idx % B;
-            const int gidx = node * q.len + pos;
-            if (gidx >= nout) continue;
-            const float acc = sum_final_values(p, q, sP, s_inj, s_final, s_touch, node, (size_t)pos * B + b);
-            const size_t oi = (size_t)b * nout + gidx;
-            p.out[oi] = finish_out(p, acc, oi);
-          }
-        }
-        if (p.rep) write_report(p, q.n_cw, s_final, s_nrm, s_rat);
-      }
     }
   }
-  if (!PAIR && p.tail_fix) {
-    // The whole (co-resident) grid waits for the word the last deciding CTA writes -- a bounded wait, about a
-    // microsecond in the usual case where nothing was detected -- and does the fix kernel's work together when
-    // some codeword needs it (with two and more parities that includes the pass over the spare parities and its
-    // grid barrier, which every CTA then takes): no second launch behind every check.
+  // No fix kernel follows a check whose sums are wanted.  The CTAs that take part stay until the CTA of the last
+  // codeword to decide has written one word (nothing to do / some codeword needs work) -- a bounded wait, about a
+  // microsecond when nothing was detected -- and in the second case do the fix kernel's work together (`fix_body`, the
+  // same code).  Small batches with at most one parity (no plan has a spare parity to be verified against, so the
+  // plans are final): the CTAs that decided the codewords, which end at about the same time anyway.  Large batches, or
+  // two and more parities: the whole (co-resident) grid; with spare parities that includes their verification pass
+  // and its grid barrier, which every CTA then takes.
+  const bool whole_grid = !PAIR && p.tail_fix;
+  const unsigned n_fix = whole_grid ? gdim : min((unsigned)q.n_cw, gdim);
+  if ((whole_grid || p.inline_fix) && bid < n_fix) {
     __shared__ unsigned s_go;
     if (tid == 0) {
       unsigned v = 0u;
@@ -1331,8 +1296,8 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
     }
     __syncthreads();
     if (s_go == 2u) {
-      if (q.r >= 2) fix_body<true>(p, q, sP, s_inj, bid, gdim);
-      else fix_body<false>(p, q, sP, s_inj, bid, gdim);
+      if (whole_grid && q.r >= 2) fix_body<true>(p, q, sP, s_inj, bid, n_fix);
+      else fix_body<false>(p, q, sP, s_inj, bid, n_fix);
     }
   }
   // every CTA read the counter before the first grid barrier
