@@ -33,10 +33,11 @@ struct CheckParams {
   float* chk;          // large batches: [unit][b][partials] of slice sum / magnitudes and checksum dot / scale
   int lazy;                // large-batch path: node outputs stay where the product kernel wrote them, only
                            // hit nodes get a working copy (set by the host together with the instantiation)
-  int inline_fix;          // the last CTA of the check kernel also recomputes the sums of located / fallen-back
-                           // nodes (small batches, at most one parity, sums wanted): no fix kernel follows
-  int tail_fix;            // large batches, at most one parity: every CTA stays until the last codeword has decided
-                           // and, if some codeword needs work, the whole grid does what the fix kernel would
+  int inline_fix;          // small batches, at most one parity, sums wanted: the CTAs that decided the codewords stay
+                           // until the last one has and, if some codeword needs work, recompute the sums of the
+                           // located / fallen-back nodes together: no fix kernel follows
+  int tail_fix;            // large batches, or two and more parities: every CTA stays until the last codeword has
+                           // decided and, if some codeword needs work, the whole grid does what the fix kernel would
   int out_act;             // forward sums: activation applied as they are written (step C1), or identity
   const float* out_mask;   // backward sums: zeroed where this input is not positive (step C2), or NULL
   uint32_t* bump;          // iteration counter of the fault plans to advance when the kernel ends, or NULL

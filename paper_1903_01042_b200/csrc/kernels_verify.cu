@@ -1,15 +1,17 @@
 // Parity-check verification of the block outputs ("General Error-Detection Method" and
 // "Decoding Algorithm" of the paper's Appendix B), soft-error injection, and the final row /
-// column sums, as two kernels (the first a cooperative launch, the second one only where it needs a barrier):
+// column sums:
 //
 //   check_kernel:  U  every (codeword, node, slice) unit: working copy of the node output
 //                     (+ injected noise), node norm, inner-checksum statistic
 //                  X  syndrome maxima, the sums s_i / c_j assuming no error, inner-checksum update
-//                  D  one CTA per codeword: thresholds, detection, location, erasure-decoding plan;
-//                     the last one writes the report
-//   fix_kernel:    returns at once unless a codeword needs work; otherwise
+//                  D  one CTA per codeword: thresholds, detection, location, erasure-decoding plan, its part
+//                     of the report; then, only if some codeword needs work (the CTAs concerned wait for that
+//                     word), the fix below inside the same launch
+//   check_pair_kernel: the backward check of one iteration and the forward check of the next, side by side
+//   fix (fix_body; fix_kernel for the stand-alone detect / decode call):
 //                  V  verifies each decoding plan against the spare parities (codes with two and more
-//                     parities; with at most one parity the kernel is a plain launch without this pass)
+//                     parities: a grid barrier)
 //                  F  recomputes the sums of the data nodes a final plan touches with corrected /
 //                     fault-free values, rewrites the report
 //
