@@ -1262,6 +1262,60 @@ def test_config3_full_size_recorded_steps_against_the_oracle(cn, orc):
         torch.cuda.set_stream(torch.cuda.default_stream())
 
 
+def test_config3_full_size_eight_steps_per_recording(cn, orc):
+    """The launch configuration bench.py times: 8192x8192 fp32, 8x8 + 1 + 1, batch 1, a pool of eight inputs, eight
+    consecutive steps in one recording (three kernels per step: encoding, sweep in alternating directions, paired
+    check), replayed three times after one plain step, p = 1e-2.  The oracle runs the same 25 iterations at full
+    size: every report and loss of every step, the outputs at the end of each replay, the weights and the code
+    invariance at the end."""
+    cfg = wl.config("c3")
+    pairs, gnet, onet = _build_net(cn, orc, cfg)
+    it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fg = [cn.make_fault(seed=cfg.seed, layer=0, mode=cn.FAULT_BERNOULLI, p=1e-2, sigma=cfg.sigma, iteration_dev=it_dev)]
+    fo = [orc.make_fault(seed=cfg.seed, layer=0, mode=orc.FAULT_BERNOULLI, p=1e-2, sigma=cfg.sigma)]
+    pool = [wl.layer_inputs(cfg, k) for k in range(8)]
+    xs = [_dev(x) for x, _ in pool]
+    ts = [_dev(t) for _, t in pool]
+    reps = cn.new_reports(2 * 8)
+    losses = torch.zeros(8, device="cuda")
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(side)
+    try:
+        cn.net_set_next_input(gnet, xs[1])
+        cn.step(gnet, xs[0], ts[0], cfg.lr, faults=fg, reps_dev=reps[:2 * cn.REPORT_BYTES], loss_dev=losses[:1])
+        lo, out_o, reps_o = onet.step(pool[0][0], pool[0][1], cfg.lr, fo, 0)
+        assert [r.decisions() for r in cn.read_reports(reps)[:2]] == [r.decisions() for r in reps_o]
+        order = [1, 2, 3, 4, 5, 6, 7, 0]
+        before = cn.launch_count()
+        graph = cn.net_capture_steps(gnet, [xs[k] for k in order], [ts[k] for k in order], cfg.lr, faults=fg,
+                                     reps_dev=reps, reps_stride=2, loss_dev=losses, loss_stride=1, X_next_dev=xs[1])
+        assert cn.launch_count() - before == 24
+        it_dev.fill_(1)
+        detected = 0
+        for r in range(3):
+            cn.net_replay(gnet, graph)
+            rg = cn.read_reports(reps)
+            lg = losses.cpu().numpy()
+            for s_, k in enumerate(order):
+                it = 1 + 8 * r + s_
+                lo, out_o, reps_o = onet.step(pool[k][0], pool[k][1], cfg.lr, fo, it)
+                assert [x.decisions() for x in rg[2 * s_:2 * s_ + 2]] == [x.decisions() for x in reps_o], it
+                assert abs(float(lg[s_]) - lo) <= 1e-4 * max(1.0, abs(lo)), it
+                for x in rg[2 * s_:2 * s_ + 2]:
+                    detected += x.n_detected_cw
+                    if any(x.injected_mask):
+                        assert x.min_margin_hit > 10.0
+                    assert x.max_margin_clean < 0.1
+            assert _rel(gnet.output(1).cpu().numpy(), out_o) <= TOL_F32, r
+        assert detected > 0
+        assert _rel(cn.decode_weights(pairs[0].g).cpu().numpy(), pairs[0].o.decode_weights()) <= 1e-4
+        assert cn.check_invariance(pairs[0].g) < 1e-5
+    finally:
+        torch.cuda.synchronize()
+        torch.cuda.set_stream(torch.cuda.default_stream())
+
+
 def _sampled_full_size_layer(cn, orc, cfg, math, tol):
     """One layer of a batched configuration at full size, two iterations with faults.  The oracle cannot
     run this size in seconds, so the run is checked on what can be computed one by one: the injection
