@@ -6,7 +6,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcodenet.so")
 SOURCES = ["codenet_api.cu", "kernels_stream.cu", "kernels_check.cu", "kernels_verify.cu", "noalloc.cu", "kernels_tc.cu"]
-HEADERS = [os.path.join(CSRC, "codenet_internal.cuh"), os.path.join(CSRC, "check_device.cuh"),
+HEADERS = [os.path.join(CSRC, "codenet_internal.cuh"), os.path.join(CSRC, "check_device.cuh"), os.path.join(CSRC, "encode_device.cuh"),
            os.path.join(os.path.dirname(HERE), "include", "codenet.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]

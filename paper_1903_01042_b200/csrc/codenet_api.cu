@@ -463,12 +463,17 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
   const int emit = (B > 8 && tc_backward_update_supported(g, L->desc.math, B)) ? (g.dtype == CODENET_F32 ? 1 : 2) : 0;
   // (a fused tensor-core sweep that shares items out among CTAs adds into Z: the encoding kernel clears it on its way)
   const bool clear_z = emit != 0 && tc_backward_update_splits(*L, B);
-  CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit, L->small.on ? &L->small : nullptr,
-                               clear_z ? L->ws.Y : nullptr, clear_z ? (size_t)g.m * g.Nn * g.b_c * B : 0));
+  const bool next = B <= 8 && lookahead_ok(L, X_next_dev, B);
+  // The step of a one-layer network with the loss folded into the encoding, a look-ahead sweep and a paired check
+  // behind it: the encoding rides on the sweep's launch instead of standing between the previous check and the sweep.
+  const bool ride = next && fuse != nullptr && fuse->defer && !L->small.on && pair != nullptr && pair_supported(*L, B);
+  if (!ride)
+    CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit, L->small.on ? &L->small : nullptr,
+                                 clear_z ? L->ws.Y : nullptr, clear_z ? (size_t)g.m * g.Nn * g.b_c * B : 0));
   int src_kind;
   if (B <= 8) {
-    const bool next = lookahead_ok(L, X_next_dev, B);
-    CN_TRY(launch_backward_update_fused(*L, B, lr, L->ws.Y, next ? X_next_dev : nullptr, g.n_in, L->ws.Ynext, st));
+    CN_TRY(launch_backward_update_fused(*L, B, lr, L->ws.Y, next ? X_next_dev : nullptr, g.n_in, L->ws.Ynext, st,
+                                        ride ? X_dev : nullptr, ride ? Delta_dev : nullptr, ride ? fuse : nullptr));
     L->next_x = next ? X_next_dev : nullptr;
     L->next_B = B;
     src_kind = 1;

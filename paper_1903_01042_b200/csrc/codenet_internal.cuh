@@ -155,8 +155,20 @@ cudaError_t launch_forward_products(const Geom& g, const float* x, int ldx, int 
 cudaError_t launch_forward_products_plain(const Geom& g, const float* x, int ldx, int B, float* Y,
                                           cudaStream_t st);   // never allocates (no profiling events)
 // xnext != NULL: also produce the next iteration's feedforward partials ynext[strip][coded row][b]
+struct LossFuse;
+// enc_fuse != NULL: the launch also carries the additional encoding of the vectors (which then is not launched on its
+// own): its CTAs write Xt, Dt, the slice sums, delta^L and the loss partials for the check that follows, and the sweep
+// forms the delta~ / x~ entries it needs itself from the sums, the target and the raw input.
 cudaError_t launch_backward_update_fused(const codenet_layer_impl& L, int B, float lr, float* zpart,
-                                         const float* xnext, int ldxn, float* ynext, cudaStream_t st);
+                                         const float* xnext, int ldxn, float* ynext, cudaStream_t st,
+                                         const float* enc_X = nullptr, const float* enc_Delta = nullptr,
+                                         const LossFuse* enc_fuse = nullptr);
+// The 16-byte path of the vector encoding needs every length, offset and pointer to be a multiple of four floats.
+inline bool encode_vec_ok(const Geom& g, const float* X, const float* Delta, const float* S, const float* target) {
+  return g.b_c % 4 == 0 && g.b_r % 4 == 0 && g.Tc % 4 == 0 && g.T % 4 == 0 && g.n_in % 4 == 0 && g.n_out % 4 == 0 &&
+         g.Mbr % 4 == 0 && (reinterpret_cast<uintptr_t>(X) & 15u) == 0 && (reinterpret_cast<uintptr_t>(Delta) & 15u) == 0 &&
+         (reinterpret_cast<uintptr_t>(S) & 15u) == 0 && (reinterpret_cast<uintptr_t>(target) & 15u) == 0;
+}
 int backward_strip_elems(int dtype);  // columns per CTA of the fused backward kernel
 cudaError_t launch_backward_products(const codenet_layer_impl& L, int B, float* Z, cudaStream_t st);
 cudaError_t launch_update(const codenet_layer_impl& L, int B, float lr, cudaStream_t st);

@@ -4,6 +4,8 @@
 // the backward pass writes each block back in the same sweep.
 #include "codenet_internal.cuh"
 
+#include <string.h>
+
 namespace codenet {
 
 unsigned long long g_launches = 0;
@@ -64,6 +66,8 @@ template <int N> __device__ __forceinline__ void load_x(const float* p, float (&
     v[4 * q] = t.x; v[4 * q + 1] = t.y; v[4 * q + 2] = t.z; v[4 * q + 3] = t.w;
   }
 }
+
+#include "encode_device.cuh"
 
 // -------------------------------------------------------------------------------------------
 // Step O1: y_ij = W~_ij x_j for every active node (i < M, j < n).  One warp owns RW coded rows
@@ -144,7 +148,8 @@ template <typename T, int BT, bool NEXT>
 __global__ void __launch_bounds__(BU_THREADS)
 backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __restrict__ Dt, int B,
                        float lr, int R, int RT, float* __restrict__ zpart,
-                       const float* __restrict__ xnext, int ldxn, float* __restrict__ ynext, int reverse, int keep_from) {
+                       const float* __restrict__ xnext, int ldxn, float* __restrict__ ynext, int reverse, int keep_from,
+                       int n_enc, EncodeArgs ea) {
   constexpr int VEC = Raw16<T>::N;
   extern __shared__ float sdelta[];  // [rows of the tile][BT], then (NEXT) [rows][4 warps][BT]
   // Tiles are walked column strip by column strip: the parity block-columns first, then the data
@@ -153,13 +158,22 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
   // touched last and finds part of it still in L2.  When this sweep is the only pass of an iteration (it takes
   // the next feedforward products as well) every other launch walks the tiles in the opposite order (reverse),
   // for the same reason: the last tiles of one sweep, updated and still in L2, are the first of the next.
+  // n_enc > 0: the first n_enc CTAs of the launch do the additional encoding of the vectors (the stand-alone
+  // kernel's code) for the check that follows, and the sweep CTAs form the delta~ and x~ entries they need
+  // themselves, from the last layer's sums, the target and the raw input, with that code's arithmetic: the
+  // encoding no longer stands between the check of one iteration and the sweep of the next.
+  if (n_enc > 0 && (int)blockIdx.x < n_enc) {
+    encode_vectors_body(g, ea, (int)blockIdx.x, n_enc);
+    return;
+  }
+  const int cta = (int)blockIdx.x - n_enc, n_sweep = (int)gridDim.x - n_enc;
   const int n_rowtiles = g.M * RT;
-  const int bx = reverse ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
-  const uint64_t pol = l2_policy((int)blockIdx.x >= keep_from);   // the last CTAs' tiles stay for the next sweep
+  const int bx = reverse ? n_sweep - 1 - cta : cta;
+  const uint64_t pol = l2_policy(cta >= keep_from);   // the last CTAs' tiles stay for the next sweep
   uint64_t pol_keep;   // the partial sums the check kernel reads next
   asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
   const int strip_order = bx / n_rowtiles, rowtile = bx % n_rowtiles;
-  const int n_strips = gridDim.x / n_rowtiles;
+  const int n_strips = n_sweep / n_rowtiles;
   const int data_strips = (g.n * g.ldb) / (BU_THREADS * VEC);  // strips wholly inside the data columns
   int strip;
   if (strip_order < n_strips - data_strips) strip = data_strips + strip_order;
@@ -169,7 +183,26 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
   const int nrows = min(R, g.b_r - r0);
   for (int idx = threadIdx.x; idx < nrows * BT; idx += BU_THREADS) {
     const int rr = idx / BT, b = idx % BT;
-    sdelta[idx] = b < B ? Dt[(size_t)b * g.Mbr + (size_t)i * g.b_r + r0 + rr] : 0.0f;
+    float d = 0.0f;
+    if (b < B && n_enc == 0) {
+      d = Dt[(size_t)b * g.Mbr + (size_t)i * g.b_r + r0 + rr];
+    } else if (b < B) {
+      // delta^L = 2 (y - s) / (N B) of the mean-squared-error loss, or the parity combination of it
+      const float* fy = ea.lf.target + (size_t)b * g.n_out;
+      const float* fs = ea.lf.S + (size_t)b * g.n_out;
+      const int e = r0 + rr;
+      if (i < g.m) {
+        const int gi = i * g.b_r + e;
+        if (gi < g.n_out) d = 2.0f * (fy[gi] - fs[gi]) * ea.lf.scale;
+      } else {
+        for (int q = 0; q < g.m; ++q) {
+          const int gi = q * g.b_r + e;
+          if (gi >= g.n_out) break;
+          d = fmaf(g.Pr[q * g.r_row + (i - g.m)], 2.0f * (fy[gi] - fs[gi]) * ea.lf.scale, d);
+        }
+      }
+    }
+    sdelta[idx] = d;
   }
   __syncthreads();
   const int gc0 = (strip * BU_THREADS + threadIdx.x) * VEC;
@@ -194,7 +227,23 @@ backward_update_kernel(Geom g, const float* __restrict__ Xt, const float* __rest
 #pragma unroll
   for (int b = 0; b < BT; ++b) {
     if (b < B) {
-      load_x<VEC>(Xt + (size_t)b * g.ld + gc0, xs[b]);
+      if (n_enc == 0) {
+        load_x<VEC>(Xt + (size_t)b * g.ld + gc0, xs[b]);
+      } else if (j < g.n) {
+        load_x<VEC>(ea.X + (size_t)b * g.n_in + gc0, xs[b]);      // (no padding between the sub-vectors here)
+      } else {
+        // x~ of a parity block-column: the combination of the data sub-vectors, in their order
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) xs[b][k] = 0.0f;
+        const int e = gc0 - j * g.ldb;
+        for (int q = 0; q < g.n; ++q) {
+          float t[VEC];
+          load_x<VEC>(ea.X + (size_t)b * g.n_in + (size_t)q * g.b_c + e, t);
+          const float c = g.Pc[q * g.r_col + (j - g.n)];
+#pragma unroll
+          for (int k = 0; k < VEC; ++k) xs[b][k] = fmaf(c, t[k], xs[b][k]);
+        }
+      }
 #pragma unroll
       for (int k = 0; k < VEC; ++k) xs[b][k] *= lr;
     } else {
@@ -451,16 +500,30 @@ cudaError_t forward_dispatch(const Geom& g, const float* x, int ldx, int B, floa
 
 template <typename T, bool NEXT>
 cudaError_t backward_fused_launch(const codenet_layer_impl& L, int B, float lr, float* zpart, const float* xnext,
-                                  int ldxn, float* ynext, cudaStream_t st) {
+                                  int ldxn, float* ynext, cudaStream_t st, const float* enc_X, const float* enc_Delta,
+                                  const LossFuse* enc_fuse) {
   constexpr int VEC = Raw16<T>::N;
   const Geom& g = L.g;
   const int bt = B > 4 ? 8 : (B > 2 ? 4 : (B > 1 ? 2 : 1));
   dim3 grid(((g.ld / VEC + BU_THREADS - 1) / BU_THREADS) * (g.M * L.bwd_rt));
+  // the additional encoding rides on this launch (its CTAs come first): see the kernel
+  EncodeArgs ea;
+  memset(&ea, 0, sizeof(ea));
+  int n_enc = 0;
+  if (enc_fuse != nullptr) {
+    ea.X = enc_X; ea.Delta = enc_Delta; ea.B = B; ea.Xt = L.ws.Xt; ea.Dt = L.ws.Dt; ea.dsum = L.ws.dsum; ea.xsum = L.ws.xsum;
+    ea.lf = *enc_fuse;
+    ea.em.dcount = (size_t)B * g.Mbr;
+    ea.vec_ok = encode_vec_ok(g, enc_X, enc_Delta, enc_fuse->S, enc_fuse->target) ? 1 : 0;
+    n_enc = (g.Nn * g.nsc + g.M * g.ns) * B;
+  }
+  const int n_sweep = (int)grid.x;
+  grid.x += n_enc;
   const size_t smem = (size_t)L.bwd_rows * bt * sizeof(float) * (NEXT ? 5 : 1);
   const float* Xt = L.ws.Xt;
   const float* Dt = L.ws.Dt;
   int reverse = 0;
-  int keep_from = (int)grid.x;   // no tile is kept
+  int keep_from = n_sweep;   // no tile is kept
   if (NEXT) {
     reverse = L.sweep_reverse; L.sweep_reverse ^= 1;
     // the last 48 MB of a sweep stay at normal priority (measured on a B200 against 0, 96 and 160 MB: larger tails
@@ -468,13 +531,13 @@ cudaError_t backward_fused_launch(const codenet_layer_impl& L, int B, float lr, 
     const size_t keep_bytes = (size_t)48 << 20;
     const size_t cta_bytes = (size_t)L.bwd_rows * BU_THREADS * 16;
     const size_t keep_ctas = keep_bytes / cta_bytes;
-    keep_from = keep_ctas >= grid.x ? 0 : (int)(grid.x - keep_ctas);
+    keep_from = keep_ctas >= (size_t)n_sweep ? 0 : (int)(n_sweep - keep_ctas);
   }
   switch (bt) {
-    case 1: backward_update_kernel<T, 1, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
-    case 2: backward_update_kernel<T, 2, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
-    case 4: backward_update_kernel<T, 4, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
-    default: backward_update_kernel<T, 8, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from); break;
+    case 1: backward_update_kernel<T, 1, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from, n_enc, ea); break;
+    case 2: backward_update_kernel<T, 2, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from, n_enc, ea); break;
+    case 4: backward_update_kernel<T, 4, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from, n_enc, ea); break;
+    default: backward_update_kernel<T, 8, NEXT><<<grid, BU_THREADS, smem, st>>>(g, Xt, Dt, B, lr, L.bwd_rows, L.bwd_rt, zpart, xnext, ldxn, ynext, reverse, keep_from, n_enc, ea); break;
   }
   count_launch();
   return cudaGetLastError();
@@ -494,14 +557,15 @@ cudaError_t launch_forward_products_plain(const Geom& g, const float* x, int ldx
 }
 
 cudaError_t launch_backward_update_fused(const codenet_layer_impl& L, int B, float lr, float* zpart,
-                                         const float* xnext, int ldxn, float* ynext, cudaStream_t st) {
+                                         const float* xnext, int ldxn, float* ynext, cudaStream_t st,
+                                         const float* enc_X, const float* enc_Delta, const LossFuse* enc_fuse) {
   ProfileScope scope(CODENET_KERNEL_BACKWARD_UPDATE, st);
   const bool bf16 = L.g.dtype == CODENET_BF16;
   if (xnext)
-    return bf16 ? backward_fused_launch<__nv_bfloat16, true>(L, B, lr, zpart, xnext, ldxn, ynext, st)
-                : backward_fused_launch<float, true>(L, B, lr, zpart, xnext, ldxn, ynext, st);
-  return bf16 ? backward_fused_launch<__nv_bfloat16, false>(L, B, lr, zpart, nullptr, 0, nullptr, st)
-              : backward_fused_launch<float, false>(L, B, lr, zpart, nullptr, 0, nullptr, st);
+    return bf16 ? backward_fused_launch<__nv_bfloat16, true>(L, B, lr, zpart, xnext, ldxn, ynext, st, enc_X, enc_Delta, enc_fuse)
+                : backward_fused_launch<float, true>(L, B, lr, zpart, xnext, ldxn, ynext, st, enc_X, enc_Delta, enc_fuse);
+  return bf16 ? backward_fused_launch<__nv_bfloat16, false>(L, B, lr, zpart, nullptr, 0, nullptr, st, nullptr, nullptr, nullptr)
+              : backward_fused_launch<float, false>(L, B, lr, zpart, nullptr, 0, nullptr, st, nullptr, nullptr, nullptr);
 }
 
 int backward_strip_elems(int dtype) { return BU_THREADS * (dtype == CODENET_BF16 ? 8 : 4); }

@@ -949,9 +949,10 @@ def test_several_steps_recorded_into_one_graph(cn, orc, lookahead):
     graph = cn.net_capture_steps(gnet, [xs[k] for k in order], [ts[k] for k in order], cfg.lr, faults=fg,
                                  reps_dev=reps, reps_stride=2, loss_dev=losses, loss_stride=1,
                                  X_next_dev=xs[1] if lookahead else None)
-    # encoding, sweep, one check for two stages -- for every step whose successor the recording knows: all five with
-    # the input after the last one announced, else the first step of a replay runs its own forward stage (sweep, check)
-    assert cn.launch_count() - before == (15 if lookahead else 17), cn.launch_count() - before
+    # two launches (the sweep, which carries the vector encoding, and one check for two stages) for every step whose
+    # successor the recording knows: all five with the input after the last one announced; else the first step of a
+    # replay also runs its own forward stage (sweep, check) and the last one is encoding, sweep and its own check
+    assert cn.launch_count() - before == (10 if lookahead else 13), cn.launch_count() - before
     it_dev.fill_(1)
     seen = set()
     for r in range(3):
@@ -1264,8 +1265,8 @@ def test_config3_full_size_recorded_steps_against_the_oracle(cn, orc):
 
 def test_config3_full_size_eight_steps_per_recording(cn, orc):
     """The launch configuration bench.py times: 8192x8192 fp32, 8x8 + 1 + 1, batch 1, a pool of eight inputs, eight
-    consecutive steps in one recording (three kernels per step: encoding, sweep in alternating directions, paired
-    check), replayed three times after one plain step, p = 1e-2.  The oracle runs the same 25 iterations at full
+    consecutive steps in one recording (two kernels per step: the sweep, in alternating directions and with the vector
+    encoding aboard, and the paired check), replayed three times after one plain step, p = 1e-2.  The oracle runs the same 25 iterations at full
     size: every report and loss of every step, the outputs at the end of each replay, the weights and the code
     invariance at the end."""
     cfg = wl.config("c3")
@@ -1290,7 +1291,7 @@ def test_config3_full_size_eight_steps_per_recording(cn, orc):
         before = cn.launch_count()
         graph = cn.net_capture_steps(gnet, [xs[k] for k in order], [ts[k] for k in order], cfg.lr, faults=fg,
                                      reps_dev=reps, reps_stride=2, loss_dev=losses, loss_stride=1, X_next_dev=xs[1])
-        assert cn.launch_count() - before == 24
+        assert cn.launch_count() - before == 16     # per step: the sweep (with the encoding aboard) and the paired check
         it_dev.fill_(1)
         detected = 0
         for r in range(3):
