@@ -466,7 +466,13 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
   const bool next = B <= 8 && lookahead_ok(L, X_next_dev, B);
   // The step of a one-layer network with the loss folded into the encoding, a look-ahead sweep and a paired check
   // behind it: the encoding rides on the sweep's launch instead of standing between the previous check and the sweep.
-  const bool ride = next && fuse != nullptr && fuse->defer && !L->small.on && pair != nullptr && pair_supported(*L, B);
+  FaultDev fd, fdn;
+  const bool inject = fill_fault(fault, &fd);
+  const bool inject_next = pair != nullptr && fill_fault(pair->fault_next, &fdn);
+  // (a layer that checks nothing can share a launch for its two sums only while nothing is to be injected)
+  const bool can_pair = pair != nullptr && next && C_dev != nullptr && pair->S_next != nullptr && pair_supported(*L, B) &&
+                        (pair_checks(*L) || (!inject && !inject_next));
+  const bool ride = can_pair && fuse != nullptr && fuse->defer && !L->small.on;
   if (!ride)
     CN_TRY(launch_encode_vectors(*L, X_dev, Delta_dev, B, st, fuse, emit, L->small.on ? &L->small : nullptr,
                                  clear_z ? L->ws.Y : nullptr, clear_z ? (size_t)g.m * g.Nn * g.b_c * B : 0));
@@ -488,11 +494,7 @@ static int backward_update_impl(codenet_layer_t* L, const float* Delta_dev, cons
     }
     src_kind = 0;
   }
-  FaultDev fd;
-  const bool inject = fill_fault(fault, &fd);
-  if (pair != nullptr && L->next_x != nullptr && C_dev != nullptr && pair->S_next != nullptr && pair_supported(*L, B)) {
-    FaultDev fdn;
-    const bool inject_next = fill_fault(pair->fault_next, &fdn);
+  if (can_pair) {
     PairNext nx;
     nx.X_next = X_next_dev; nx.fault = inject_next ? &fdn : nullptr; nx.S_next = pair->S_next; nx.rep_next = pair->rep_next;
     nx.commit_S = pair->commit_S; nx.commit_S_to = pair->commit_S_to; nx.commit_n = pair->commit_n;

@@ -231,6 +231,7 @@ struct PairNext {
   const float* loss_partials; int loss_n; float* loss_out;   // a loss whose partial sums wait to be added up, or NULL
 };
 bool pair_supported(const codenet_layer_impl& L, int B);
+bool pair_checks(const codenet_layer_impl& L);   // the pair is the cooperative check kernel (else: the two plain sums)
 cudaError_t launch_check_pair(const codenet_layer_impl& L, const float* src, float* Yw, const float* Delta, int B,
                               const FaultDev* fault, float* out, float lr, codenet_report_t* rep,
                               const PairNext& nx, cudaStream_t st);

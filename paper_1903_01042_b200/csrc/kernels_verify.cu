@@ -1481,32 +1481,66 @@ __global__ void __launch_bounds__(256) input_fault_kernel(Geom g, SmallDev sf, i
 // Plain sums of the data-node outputs for calls that check nothing (no code, or the checks switched off, and no
 // injection): s_i = sum_j y_ij / c_j = sum_i z_ij straight from the node outputs or their partial sums, in the same
 // fixed order as the checked path, an empty report.  No barrier, no working copy, no inner-checksum update.
-__global__ void __launch_bounds__(CK_THREADS) sum_outputs_kernel(CheckParams p) {
+// bid / gdim: the CTA's index and the number of CTAs within its part (a launch of its own: the whole grid).
+__device__ __forceinline__ void sum_body(const CheckParams& p, const unsigned bid, const unsigned gdim) {
   const Geom& g = p.g;
   const bool fwd = p.phase == CODENET_PHASE_FWD;
   const PhaseGeom q = phase_geom(g, p.phase, p.B);
   const int B = p.B;
   const int nout = fwd ? g.n_out : g.n_in;
-  for (size_t idx = blockIdx.x * (size_t)CK_THREADS + threadIdx.x; idx < (size_t)nout * B;
-       idx += (size_t)gridDim.x * CK_THREADS) {
+  for (size_t idx = bid * (size_t)CK_THREADS + threadIdx.x; idx < (size_t)nout * B; idx += (size_t)gdim * CK_THREADS) {
     const int b = (int)(idx % B), gidx = (int)(idx / B);
     int node, pos;
     output_index(g, fwd, gidx, &node, &pos);
     float acc = 0.0f;
     for (int cw = 0; cw < q.n_cw; ++cw) acc += clean_value(p, q, cw, node, (size_t)pos * B + b);
     const size_t oi = (size_t)b * nout + gidx;
+    // (paired form: what the previous pair staged at this index goes out first, by the thread that overwrites it)
+    if (p.commit_S != nullptr && oi < (size_t)p.commit_n) p.commit_S_to[oi] = p.commit_S[oi];
     p.out[oi] = finish_out(p, acc, oi);
   }
   codenet_report_t* rep = p.rep;
-  if (rep && blockIdx.x == 0) {
-    if (threadIdx.x == 0) {
-      rep->status = (p.tc_flag && *p.tc_flag) ? (uint32_t)CODENET_TIMEOUT : (uint32_t)CODENET_CLEAN;
-      rep->n_detected_cw = 0; rep->n_flagged_nodes = 0; rep->n_fallback_cw = 0;
-      rep->detected_mask = 0; rep->min_margin_hit = FLT_MAX; rep->max_margin_clean = 0.0f;
+  if (bid == 0) {
+    if (p.commit_rep != nullptr) {
+      const uint32_t* from = reinterpret_cast<const uint32_t*>(p.commit_rep);
+      uint32_t* to = reinterpret_cast<uint32_t*>(p.commit_rep_to);
+      for (int t = threadIdx.x; t < (int)(sizeof(codenet_report_t) / sizeof(uint32_t)); t += CK_THREADS) to[t] = from[t];
+      __syncthreads();
     }
-    for (int cw = threadIdx.x; cw < MAXN; cw += CK_THREADS) { rep->flagged_mask[cw] = 0; rep->injected_mask[cw] = 0; }
+    if (rep) {
+      if (threadIdx.x == 0) {
+        rep->status = (p.tc_flag && *p.tc_flag) ? (uint32_t)CODENET_TIMEOUT : (uint32_t)CODENET_CLEAN;
+        rep->n_detected_cw = 0; rep->n_flagged_nodes = 0; rep->n_fallback_cw = 0;
+        rep->detected_mask = 0; rep->min_margin_hit = FLT_MAX; rep->max_margin_clean = 0.0f;
+      }
+      for (int cw = threadIdx.x; cw < MAXN; cw += CK_THREADS) { rep->flagged_mask[cw] = 0; rep->injected_mask[cw] = 0; }
+    }
   }
-  if (p.bump != nullptr && blockIdx.x == 0 && threadIdx.x == 0) *p.bump += 1u;
+  if (p.loss_partials != nullptr && bid == gdim - 1) {
+    // the step's loss from the partial sums the vector encoding left (its own order: see check_body)
+    __shared__ float red[CK_WARPS];
+    float t = 0.0f;
+    if (threadIdx.x < 128)
+      for (int idx = threadIdx.x; idx < p.loss_n; idx += 128) t += __ldcg(&p.loss_partials[idx]);
+    t = warp_sum(t);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = t;
+    __syncthreads();
+    if (threadIdx.x == 0) *p.loss_out = red[0] + red[1] + red[2] + red[3];
+  }
+  if (p.bump != nullptr && bid == 0 && threadIdx.x == 0) *p.bump += 1u;
+}
+
+__global__ void __launch_bounds__(CK_THREADS) sum_outputs_kernel(CheckParams p) {
+  sum_body(p, blockIdx.x, gridDim.x);
+}
+
+// The sums of one iteration's backward stage and of the next iteration's forward stage in one plain launch, for
+// layers that check nothing: the counterpart of check_pair_kernel (same staging of the next iteration's sums and
+// report, same loss hand-over), without a barrier: every output is written by one thread.
+__global__ void __launch_bounds__(CK_THREADS) sum_pair_kernel(const __grid_constant__ PairParams pp) {
+  const int part = blockIdx.x >= (unsigned)pp.n_first ? 1 : 0;
+  const CheckParams& p = pp.v[part];
+  sum_body(p, part ? blockIdx.x - pp.n_first : blockIdx.x, part ? gridDim.x - pp.n_first : pp.n_first);
 }
 
 int g_coop_blocks_check = 0, g_coop_blocks_fix = 0, g_coop_blocks_check_max = 0;
@@ -1571,10 +1605,20 @@ void fill_check_params(const codenet_layer_impl& L, int phase, const float* src,
 }
 }  // namespace
 
-bool pair_supported(const codenet_layer_impl& L, int B) {
+// Both checks of a layer decide something (node check, at most one parity per code: the cooperative pair) ...
+bool pair_checks(const codenet_layer_impl& L) {
   const Geom& g = L.g;
-  return L.pair_ok && B == 1 && g.locate_mode == CODENET_LOCATE_NODECHECK && g.r_row <= 1 && g.r_col <= 1 &&
-         !L.small.on && keeps_checksums(g);
+  return g.locate_mode == CODENET_LOCATE_NODECHECK && g.r_row <= 1 && g.r_col <= 1 && keeps_checksums(g);
+}
+// ... or neither does anything but sum (checks switched off, or no code and no node check: the plain pair, which
+// cannot inject faults).
+static bool pair_sums_only(const codenet_layer_impl& L) {
+  const Geom& g = L.g;
+  return (g.locate_mode == CODENET_LOCATE_OFF ||
+          (g.r_row == 0 && g.r_col == 0 && g.locate_mode != CODENET_LOCATE_NODECHECK)) && !keeps_checksums(g);
+}
+bool pair_supported(const codenet_layer_impl& L, int B) {
+  return L.pair_ok && B == 1 && !L.small.on && (pair_checks(L) || pair_sums_only(L));
 }
 
 cudaError_t launch_check_pair(const codenet_layer_impl& L, const float* src, float* Yw, const float* Delta, int B,
@@ -1599,6 +1643,18 @@ cudaError_t launch_check_pair(const codenet_layer_impl& L, const float* src, flo
   pf.commit_rep = nx.commit_rep; pf.commit_rep_to = nx.commit_rep_to;
   pf.loss_partials = nx.loss_partials; pf.loss_n = nx.loss_n; pf.loss_out = nx.loss_out;
   if (L.bump_after != nullptr) { pb.bump = L.bump_after; L.bump_done = true; }
+  if (!pair_checks(L)) {
+    // nothing to inject and nothing to decide (the caller has made sure of the first): the two sums, one plain launch
+    size_t nb = ((size_t)g.n_in * B + CK_THREADS - 1) / CK_THREADS, nf = ((size_t)g.n_out * B + CK_THREADS - 1) / CK_THREADS;
+    if (nb > 148 * 4) nb = 148 * 4;
+    if (nf > 148 * 4) nf = 148 * 4;
+    if (nb < 1) nb = 1;
+    if (nf < 2) nf = 2;
+    pp.n_first = (int)nb;
+    sum_pair_kernel<<<(unsigned)(nb + nf), CK_THREADS, 0, st>>>(pp);
+    count_launch();
+    return cudaGetLastError();
+  }
   // forward part: one warp per unit and one thread per element; backward part: the same and a warp per checksum
   // vector, within what is left of the co-resident limit
   const size_t cap = (size_t)g_coop_blocks_check;
