@@ -57,9 +57,8 @@ struct CheckStats {
   unsigned ratio[CODENET_MAX_NODES * CODENET_MAX_NODES];  // [codeword][node] inner-check statistic / threshold
   unsigned syn[CODENET_MAX_NODES];                        // [codeword] max |syndrome|
   unsigned resid[CODENET_MAX_NODES];                      // [codeword] max residual of the decoding plan
-  unsigned need_fix, done_d;
-  unsigned fix_go;   // written by the CTA of the last codeword to decide: 1 = no codeword needs work, 2 = some do
-  unsigned pad_;
+  unsigned need_fix;   // some codeword needs work (read by a fix kernel that follows)
+  unsigned done_d;     // low half: codewords that have decided; high half: how many of them need work
 };
 
 // Per-codeword decision and erasure-decoding plan.

@@ -477,7 +477,6 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
   __shared__ unsigned long long s_F;
   __shared__ float s_tau, s_scale, s_smax, s_h;
   __shared__ float s_nrm[MAXN], s_rat[MAXN];
-  __shared__ int s_last;
 
   for (int t = tid; t < q.kd * q.r; t += CK_THREADS) sP[t] = q.P[t];
   for (int t = tid; t < MAXN; t += CK_THREADS) s_syn[t] = 0u;
@@ -1253,31 +1252,20 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
         atomicMin(reinterpret_cast<unsigned*>(&r->min_margin_hit), __float_as_uint(cw_min_hit));
         atomicMax(reinterpret_cast<unsigned*>(&r->max_margin_clean), __float_as_uint(cw_max_clean));
       }
-      s_last = 0;
       if (p.inline_fix || p.tail_fix) {
-        // only the in-kernel fix needs to know which CTA comes last; the same counter carries, above bit 16,
-        // how many codewords need work, so the last CTA learns both from one atomic
+        // one counter tells the waiting CTAs both things: how many codewords have decided (low half) and how many of
+        // them need work (high half)
         __threadfence();
-        const unsigned add = 1u + (state != 0 ? 0x10000u : 0u);
-        const unsigned done = atomicAdd(&p.st->done_d, add);
-        if ((done & 0xFFFFu) == (unsigned)q.n_cw - 1) s_last = ((done + add) >> 16) != 0u ? 2 : 1;
+        atomicAdd(&p.st->done_d, 1u + (state != 0 ? 0x10000u : 0u));
       } else if (state != 0) {
         atomicOr(&p.st->need_fix, 1u);   // read by the fix kernel that follows
       }
     }
     __syncthreads();
-    if (s_last) {
-      // every plan is written: tell the waiting CTAs whether there is anything to do
-      if (tid == 0) {
-        __threadfence();
-        atomicExch(&p.st->fix_go, (unsigned)s_last);
-      }
-    }
   }
-  // No fix kernel follows a check whose sums are wanted.  The CTAs that take part stay until the CTA of the last
-  // codeword to decide has written one word (nothing to do / some codeword needs work) -- a bounded wait, about a
-  // microsecond when nothing was detected -- and in the second case do the fix kernel's work together (`fix_body`, the
-  // same code).  Small batches with at most one parity (no plan has a spare parity to be verified against, so the
+  // No fix kernel follows a check whose sums are wanted.  The CTAs that take part stay until the counter says that
+  // every codeword has decided (a bounded wait, about a microsecond) and, if it also says that some codeword needs
+  // work, do the fix kernel's work together (`fix_body`, the same code).  Small batches with at most one parity (no plan has a spare parity to be verified against, so the
   // plans are final): the CTAs that decided the codewords, which end at about the same time anyway.  Large batches, or
   // two and more parities: the whole (co-resident) grid; with spare parities that includes their verification pass
   // and its grid barrier, which every CTA then takes.
@@ -1286,15 +1274,15 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
   if ((whole_grid || p.inline_fix) && bid < n_fix) {
     __shared__ unsigned s_go;
     if (tid == 0) {
-      unsigned v = 0u;
+      unsigned v = 0u, go = 0u;
       for (unsigned spin = 0; spin < (1u << 22); ++spin) {
-        v = *reinterpret_cast<volatile unsigned*>(&p.st->fix_go);
-        if (v != 0u) break;
+        v = *reinterpret_cast<volatile unsigned*>(&p.st->done_d);
+        if ((v & 0xFFFFu) >= (unsigned)q.n_cw) { go = (v >> 16) != 0u ? 2u : 1u; break; }
         __nanosleep(64);
       }
-      if (v == 0u) atomicExch(const_cast<int*>(p.tc_flag), 1);   // gave up: reported as TIMEOUT by the next check
+      if (go == 0u) atomicExch(const_cast<int*>(p.tc_flag), 1);   // gave up: reported as TIMEOUT by the next check
       __threadfence();
-      s_go = v;
+      s_go = go;
     }
     __syncthreads();
     if (s_go == 2u) {
