@@ -663,7 +663,7 @@ def main():
                        "unit": "layer-iterations/s",
                        "h2d_bytes_per_step": bi, "d2h_bytes_per_step": bo,
                        "note": "every step: one pinned upload of [next input | target], the step, one download of "
-                               "[reports | loss]; eight steps and their copies are captured in one graph of the "
+                               "[reports | loss]; up to forty steps and their copies are captured in one graph of the "
                                "caller's (uploads and downloads on streams of their own), the host reads a replay's "
                                "losses from pinned memory after it has queued the next replay"
                                if not args.no_graphs else
