@@ -228,6 +228,7 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
     """Returns (seconds for `steps` steps, kernel launches in the timed region)."""
     L = len(layers)
     pool = 8
+    cn.net_set_lookahead(net, bool(lookahead))
     total = warmup + steps
     its = torch.arange(total, dtype=torch.int32, device="cuda")
     mode = {"bernoulli": 1, "exactly_one": 2, "none": 0}[cfg.fault_mode] if inject else 0

@@ -282,6 +282,12 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
  * its sums and report appear where this interface says when that step ends).  One-shot: cleared by that step. */
 int codenet_net_set_next_input(codenet_net_t* net, const float* X_next_dev);
 
+/* Switch the use of announced next inputs on (the default) or off.  Off: codenet_net_set_next_input and the
+ * successor inputs a recording knows are ignored, every step sweeps the weights for its own forward products (three
+ * passes over the first layer's weights per iteration instead of two).  Results are the same either way.
+ * Errors: BADARG. */
+int codenet_net_set_lookahead(codenet_net_t* net, int on);
+
 /* Give the network an iteration counter of its own (a device word, e.g. the one the fault plans read): every
  * codenet_step from now on ends by adding one to it, in its last kernel where that kernel can (so a step the caller
  * captures into a graph of their own draws a new fault pattern at every replay, like the recorded steps below).

@@ -90,6 +90,8 @@ def lib():
     L.codenet_backward_update_forward_next.argtypes = [vp, vp, vp, ip, fl, C.POINTER(Fault), vp, vp, vp,
                                                        C.POINTER(Fault), vp, vp, vp]
     L.codenet_net_set_next_input.argtypes = [vp, vp]
+    L.codenet_net_set_lookahead.argtypes = [vp, ip]
+    L.codenet_net_set_lookahead.restype = ip
     L.codenet_net_set_iteration_counter.argtypes = [vp, vp]
     L.codenet_net_set_iteration_counter.restype = ip
     L.codenet_net_capture_step.argtypes = [vp, vp, vp, ip, fl, C.POINTER(Fault), vp, vp, vp, vp, C.POINTER(ip)]
@@ -349,6 +351,11 @@ def net_create(layers, activation=ACT_IDENTITY, loss=LOSS_MSE_MEAN):
 def net_set_next_input(net, X_next_dev):
     """codenet_net_set_next_input: announce the next step's input (kept alive by the caller)."""
     _check(lib().codenet_net_set_next_input(net.h, _ptr(X_next_dev)))
+
+
+def net_set_lookahead(net, on):
+    """codenet_net_set_lookahead: use (default) or ignore announced next inputs."""
+    _check(lib().codenet_net_set_lookahead(net.h, 1 if on else 0))
 
 
 def net_set_iteration_counter(net, counter_dev):

@@ -17,6 +17,7 @@ struct codenet_net {
   float* s_stage;          // one-layer networks: sums of the next step's forward stage, done ahead by a paired check
   codenet_report_t* rep_stage;   // its report, until the step it belongs to ends
   uint32_t* step_counter;  // device word every codenet_step advances when it ends (codenet_net_set_iteration_counter), or NULL
+  int lookahead;           // 0: announced next inputs are ignored (every step runs its own forward sweep)
   float* delta[2];         // ping-pong error vectors, (B, widest layer)
   float* loss_partials;    // 512 partial sums + one counter word (loss kernel), then LOSS_FUSE_PARTIALS + a counter (loss folded into the vector encoding)
   std::vector<cudaGraphExec_t> graphs;  // captured steps (codenet_net_capture_step)
@@ -665,6 +666,7 @@ int codenet_net_create(codenet_layer_t** layers, int L, int activation, int loss
   net->s_stage = nullptr;
   net->rep_stage = nullptr;
   net->step_counter = nullptr;
+  net->lookahead = 1;
   net->x_next = nullptr;
   net->delta[0] = net->delta[1] = nullptr;
   net->loss_partials = nullptr;
@@ -712,6 +714,7 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
   if (!net || !X_dev || !target_dev || B < 1 || B > net->batch_max) return CODENET_E_BADARG;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   const int L = net->L;
+  if (!net->lookahead) net->x_next = nullptr;
   // The first layer's forward stage may have been done by the previous step (its check shared a launch with that
   // step's last backward check): its sums are in place (in the staging buffer for a one-layer network), its report
   // is staged.  And this step may end the same way for the next input.
@@ -805,6 +808,13 @@ int codenet_step(codenet_net_t* net, const float* X_dev, const void* target_dev,
     L0->bump_done = false;
     if (!bumped) CN_TRY(launch_bump_counter(net->step_counter, st));
   }
+  return CODENET_OK;
+}
+
+int codenet_net_set_lookahead(codenet_net_t* net, int on) {
+  if (!net) return CODENET_E_BADARG;
+  net->lookahead = on ? 1 : 0;
+  if (!on) net->x_next = nullptr;
   return CODENET_OK;
 }
 

@@ -920,7 +920,7 @@ def test_recorded_steps_replay_like_plain_steps(cn, orc, lookahead):
     torch.cuda.set_stream(torch.cuda.default_stream())
 
 
-@pytest.mark.parametrize("lookahead", [False, True])
+@pytest.mark.parametrize("lookahead", [False, True, "off"])
 def test_several_steps_recorded_into_one_graph(cn, orc, lookahead):
     """Five consecutive steps over a pool of five inputs recorded into one graph (each with its own reports and loss
     slot), replayed three times after one plain step.  Inside the recording every step knows its successor's input,
@@ -928,6 +928,13 @@ def test_several_steps_recorded_into_one_graph(cn, orc, lookahead):
     announced as well, that holds across the end of a replay too.  Against the oracle stepping normally."""
     cfg = wl.Config("one", [wl.LayerSpec(1024, 2048, 2, 4, 1, 1)], 1, 0.01, 16, p=0.1, seed=9)
     pairs, gnet, onet = _build_net(cn, orc, cfg)
+    if lookahead == "off":
+        # announced inputs are ignored: every step sweeps the weights for its own forward products
+        cn.net_set_lookahead(gnet, False)
+        lookahead = False
+        expected_launches = 25                        # forward sweep, check, encoding, update sweep, check
+    else:
+        expected_launches = 10 if lookahead else 13
     it_dev = torch.zeros(1, dtype=torch.int32, device="cuda")
     fg = [cn.make_fault(seed=3, layer=0, mode=cn.FAULT_BERNOULLI, p=cfg.p, sigma=10.0, iteration_dev=it_dev)]
     fo = [orc.make_fault(seed=3, layer=0, mode=orc.FAULT_BERNOULLI, p=cfg.p, sigma=10.0)]
@@ -952,7 +959,7 @@ def test_several_steps_recorded_into_one_graph(cn, orc, lookahead):
     # two launches (the sweep, which carries the vector encoding, and one check for two stages) for every step whose
     # successor the recording knows: all five with the input after the last one announced; else the first step of a
     # replay also runs its own forward stage (sweep, check) and the last one is encoding, sweep and its own check
-    assert cn.launch_count() - before == (10 if lookahead else 13), cn.launch_count() - before
+    assert cn.launch_count() - before == expected_launches, cn.launch_count() - before
     it_dev.fill_(1)
     seen = set()
     for r in range(3):
