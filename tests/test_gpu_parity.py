@@ -681,6 +681,20 @@ def test_paired_checks_in_a_network_with_hidden_layers(cn, orc):
     assert with_pairs < cn.launch_count() - launches - 39     # a forward sweep and a check launch fewer per step
 
 
+def test_paired_checks_with_the_loss_folded_into_another_layers_encoding(cn, orc):
+    """Two layers, ReLU, mean-squared-error loss, batch 1, the next input announced: the loss partials are left by the
+    LAST layer's vector encoding and added up by the paired check of the FIRST layer at the end of the step."""
+    cfg = wl.Config("two", [wl.LayerSpec(256, 1024, 2, 2, 1, 1), wl.LayerSpec(128, 256, 2, 2, 1, 1)], 1, 0.01, 30,
+                    activation="relu", loss="mse", p=3e-2, seed=7)
+    launches = cn.launch_count()
+    stats = _run_config(cn, orc, cfg, 30, TOL_F32, 1e-4, lookahead=True)
+    with_pairs = cn.launch_count() - launches
+    assert stats["corrected"] > 0
+    launches = cn.launch_count()
+    _run_config(cn, orc, cfg, 30, TOL_F32, 1e-4, lookahead=False)
+    assert with_pairs < cn.launch_count() - launches - 29
+
+
 def test_config2_mlp_relu_softmax(cn, orc):
     """784-1000-1000-10 MLP, 4x4 + 1 + 1 per layer, batch 1; error rate raised so that 200
     iterations see faults in every layer."""
