@@ -695,6 +695,48 @@ def test_paired_checks_with_the_loss_folded_into_another_layers_encoding(cn, orc
     assert with_pairs < cn.launch_count() - launches - 29
 
 
+@pytest.mark.parametrize("coded", [True, False])
+def test_layers_that_check_nothing_share_one_launch_for_their_sums(cn, orc, coded):
+    """Checks switched off (with and without parity blocks), no faults, the next input announced: the sums of a step's
+    backward stage and of the next step's forward stage come from one plain launch, the vector encoding rides on the
+    sweep (two launches per step); outputs, loss and weights as the oracle's, eagerly and through a recording."""
+    r = 1 if coded else 0
+    cfg = wl.Config("off", [wl.LayerSpec(1024, 2048, 2, 4, r, r)], 1, 0.01, 12, fault_mode="none", seed=13)
+    pairs, gnet, onet = _build_net(cn, orc, cfg, locate_mode=3)      # CODENET_LOCATE_OFF
+    pool = [wl.layer_inputs(cfg, k) for k in range(4)]
+    xs = [_dev(x) for x, _ in pool]
+    ts = [_dev(t) for _, t in pool]
+    losses = torch.zeros(4, device="cuda")
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(side)
+    try:
+        it = 0
+        for k in range(4):                                   # eager steps with the next input announced
+            cn.net_set_next_input(gnet, xs[(k + 1) % 4])
+            before = cn.launch_count()
+            cn.step(gnet, xs[k], ts[k], cfg.lr, loss_dev=losses[:1])
+            if k > 0:
+                assert cn.launch_count() - before == 2       # sweep (+ encoding), one launch for both sums
+            lo, out_o, _ = onet.step(pool[k][0], pool[k][1], cfg.lr, None, it)
+            assert _rel(gnet.output(1).cpu().numpy(), out_o) <= TOL_F32, it
+            assert abs(float(losses[0].item()) - lo) <= 1e-4 * max(1.0, abs(lo)), it
+            it += 1
+        graph = cn.net_capture_steps(gnet, xs, ts, cfg.lr, loss_dev=losses, loss_stride=1, X_next_dev=xs[0])
+        for rep_ in range(2):
+            cn.net_replay(gnet, graph)
+            lg = losses.cpu().numpy()
+            for k in range(4):
+                lo, out_o, _ = onet.step(pool[k][0], pool[k][1], cfg.lr, None, it)
+                assert abs(float(lg[k]) - lo) <= 1e-4 * max(1.0, abs(lo)), it
+                it += 1
+            assert _rel(gnet.output(1).cpu().numpy(), out_o) <= TOL_F32, rep_
+        assert _rel(cn.decode_weights(pairs[0].g).cpu().numpy(), pairs[0].o.decode_weights()) <= 1e-4
+    finally:
+        torch.cuda.synchronize()
+        torch.cuda.set_stream(torch.cuda.default_stream())
+
+
 def test_config2_mlp_relu_softmax(cn, orc):
     """784-1000-1000-10 MLP, 4x4 + 1 + 1 per layer, batch 1; error rate raised so that 200
     iterations see faults in every layer."""
