@@ -782,6 +782,18 @@ def test_config4_scaled_bf16_gaussian_code(cn, orc):
     assert stats["detected"] > 0
 
 
+def test_bfloat16_blocks_at_batch_1_with_the_encoding_aboard_the_sweep(cn, orc):
+    """bfloat16 storage, checksum code, batch 1, mean-squared-error loss, the next input announced: the streaming sweep
+    takes the next products, carries the vector encoding and is followed by the paired check (two launches per step)."""
+    cfg = wl.Config("b16", [wl.LayerSpec(2048, 2048, 2, 2, 1, 1)], 1, 0.01, 24, bf16=True, p=5e-2, seed=17)
+    launches = cn.launch_count()
+    stats = _run_config(cn, orc, cfg, 24, TOL_LOWP, 2e-3, weight_norm="fro", lookahead=True)
+    assert stats["corrected"] > 0
+    # the first step runs its own forward stage (sweep, check), encoding, sweep and pair: 5; the other 23: 2 each,
+    # the decoded-weights / report helpers launch nothing that is counted here
+    assert cn.launch_count() - launches <= 5 + 2 * 23 + 8
+
+
 # ---------------------------------------------------------------------------------------------
 # tensor-core tiles (batch >= 64)
 # ---------------------------------------------------------------------------------------------
