@@ -407,16 +407,36 @@ __device__ __forceinline__ void output_index(const Geom& g, bool fwd, int gidx, 
 }
 
 
-// Value of data node `node` of codeword `cw` at element e after decoding / fallback.
+// Value of data node `node` of codeword `cw` at element e after decoding / fallback (plans: a copy in shared memory).
 __device__ __forceinline__ float final_value(const CheckParams& p, const PhaseGeom& q, const float* sP,
-                                             const unsigned long long* s_inj, const unsigned* s_final, int cw,
-                                             int node, size_t e) {
+                                             const unsigned long long* s_inj, const unsigned* s_final,
+                                             const CwPlan* plans, int cw, int node, size_t e) {
   const CwView yw = cw_view(p, q, s_inj, cw);
   const int state = (int)s_final[cw];
   if (state == 0 || state == 4) return yw.at(q, node, e);   // (4: the verification steps disagreed: left as it is)
   if (state == 1) {
-    const CwPlan& pl = p.plan[cw];
+    const CwPlan& pl = plans[cw];
     if (!((pl.F >> node) & 1ull)) return yw.at(q, node, e);
+    if (pl.nfd == 1) {
+      // One located data node, the usual case, in few instructions (this code runs once in a while, so what it costs
+      // is the fetching of its instructions): the same operations in the same order as the general decoding below.
+      const unsigned long long F = pl.F;
+      const int qa = pl.q[0];
+      double rhs = (double)yw.at(q, q.kd + qa, e);
+#pragma unroll 1
+      for (int k0 = 0; k0 < q.kd; k0 += 8) {
+        float o8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) o8[u] = yw.at(q, min(k0 + u, q.kd - 1), e);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int k = k0 + u;
+          if (k >= q.kd || ((F >> k) & 1ull)) continue;
+          rhs -= (double)sP[k * q.r + qa] * (double)o8[u];
+        }
+      }
+      return (float)(pl.ainv[0] * rhs);
+    }
     float fix[MAXR];
     double par[MAXR];
     decode_at(yw, q, sP, pl, e, fix, par);
@@ -432,28 +452,40 @@ __device__ __forceinline__ float final_value(const CheckParams& p, const PhaseGe
 }
 
 // Sum over the codewords of one output (data node `node`, element e) with final values, in codeword order.  The values
-// of the codewords whose plan does not touch the node (the many) are plain loads, taken eight at a time so that they
-// are in flight together; s_touch[c] holds the nodes codeword c's final plan replaces (decoded or fault-free).
+// of the codewords whose plan does not touch the node (the many) are plain loads, sixteen at a time so that they are in
+// flight together; the loads of a touched codeword's decoding follow them at once (the plan sits in shared memory, so
+// nothing they need is still on its way).  s_touch[c] holds the nodes codeword c's final plan replaces (decoded or
+// fault-free).
 __device__ __forceinline__ float sum_final_values(const CheckParams& p, const PhaseGeom& q, const float* sP,
                                                   const unsigned long long* s_inj, const unsigned* s_final,
-                                                  const unsigned long long* s_touch, int node, size_t e) {
+                                                  const unsigned long long* s_touch, const CwPlan* plans, int node,
+                                                  size_t e) {
   float acc = 0.0f;
-  for (int c0 = 0; c0 < q.n_cw; c0 += 8) {
-    float v[8];
+  for (int c0 = 0; c0 < q.n_cw; c0 += 16) {
+    float v[16];
+    if (!lazy_copy(p)) {
+      // every node output sits in the working copy: one base and one stride (few instructions: see final_value)
+      const float* base = p.Yw + (size_t)node * q.n_el + e;
+      const size_t stride = (size_t)q.K * q.n_el;
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int c = min(c0 + u, q.n_cw - 1);
-      v[u] = cw_view(p, q, s_inj, c).at(q, node, e);
-    }
+      for (int u = 0; u < 16; ++u) v[u] = base[(size_t)min(c0 + u, q.n_cw - 1) * stride];
+    } else {
 #pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const int c = c0 + u;
-      if (c < q.n_cw) {
-        if ((s_touch[c] >> node) & 1ull) v[u] = final_value(p, q, sP, s_inj, s_final, c, node, e);
-        acc += v[u];
+      for (int u = 0; u < 16; ++u) {
+        const int c = min(c0 + u, q.n_cw - 1);
+        v[u] = cw_view(p, q, s_inj, c).at(q, node, e);
       }
     }
+#pragma unroll 1
+    for (int c = c0; c < min(c0 + 16, q.n_cw); ++c) {
+      if (!((s_touch[c] >> node) & 1ull)) continue;
+      const float d = final_value(p, q, sP, s_inj, s_final, plans, c, node, e);
+#pragma unroll
+      for (int u = 0; u < 16; ++u) v[u] = (c0 + u == c) ? d : v[u];
+    }
+#pragma unroll
+    for (int u = 0; u < 16; ++u)
+      if (c0 + u < q.n_cw) acc += v[u];
   }
   return acc;
 }
-

@@ -446,7 +446,7 @@ __device__ __forceinline__ void checksum_dot(const float* a, const float* w, int
 
 template <bool SPARE>
 __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, const float* sP, const unsigned long long* s_inj,
-                                         const unsigned bid, const unsigned gdim);
+                                         CwPlan* s_plan, const unsigned bid, const unsigned gdim);
 
 // PAIR: the body runs as one part of a paired launch (p.pair says which); bid / gdim are the CTA's index and the
 // number of CTAs within its part.  Both parts pass the same two grid barriers.
@@ -477,6 +477,9 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
   __shared__ unsigned long long s_F;
   __shared__ float s_tau, s_scale, s_smax, s_h;
   __shared__ float s_nrm[MAXN], s_rat[MAXN];
+  // one buffer, two tenants that never overlap in time: the tiles of the large-batch sums pass, and the plans of the fix
+  constexpr size_t kSumsBytes = sizeof(float) * BIG_KD * BIG_TR * 33, kPlanBytes = sizeof(CwPlan) * MAXN;
+  __shared__ __align__(16) unsigned char s_scratch[BIG ? (kSumsBytes > kPlanBytes ? kSumsBytes : kPlanBytes) : kPlanBytes];
 
   for (int t = tid; t < q.kd * q.r; t += CK_THREADS) sP[t] = q.P[t];
   for (int t = tid; t < MAXN; t += CK_THREADS) s_syn[t] = 0u;
@@ -818,7 +821,7 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
       if (s_syn[cw]) atomicMax(&p.st->syn[cw], s_syn[cw]);
   }
   if (big_batch && one_pass) {
-    __shared__ float s_sums[BIG_KD][BIG_TR][33];
+    float (*s_sums)[BIG_TR][33] = reinterpret_cast<float (*)[BIG_TR][33]>(s_scratch);   // [BIG_KD][BIG_TR][33]
     if (q.kd <= 8) {
       float (*s_wide)[32][33] = reinterpret_cast<float (*)[32][33]>(&s_sums[0][0][0]);   // [8][32][33]: the same bytes
       if (q.kd <= 4 && q.r <= 2) big_phase_x_wide<4, 2, 2>(p, q, sP, s_inj, s_syn, s_wide, check_off);
@@ -1215,7 +1218,12 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
           for (int t = 0; t < q.r && nq < nfd; ++t) if (!((F >> (q.kd + t)) & 1ull)) pl.q[nq++] = t;
           if (nq < nfd) ok = 0;
         }
-        if (ok && nfd > 0) {
+        if (ok && nfd == 1) {
+          // one located data node, the usual case: the 1 x 1 system as the general elimination would solve it
+          const double a00 = (double)sP[pl.fd[0] * q.r + pl.q[0]];
+          if (a00 == 0.0) ok = 0;
+          else pl.ainv[0] = 1.0 / a00;
+        } else if (ok && nfd > 0) {
           double A[MAXR * MAXR];
           for (int a = 0; a < nfd; ++a)
             for (int b = 0; b < nfd; ++b) A[a * nfd + b] = (double)sP[pl.fd[b] * q.r + pl.q[a]];
@@ -1286,8 +1294,9 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
     }
     __syncthreads();
     if (s_go == 2u) {
-      if (whole_grid && q.r >= 2) fix_body<true>(p, q, sP, s_inj, bid, n_fix);
-      else fix_body<false>(p, q, sP, s_inj, bid, n_fix);
+      CwPlan* s_plan = reinterpret_cast<CwPlan*>(s_scratch);   // (the sums pass is long over)
+      if (whole_grid && q.r >= 2) fix_body<true>(p, q, sP, s_inj, s_plan, bid, n_fix);
+      else fix_body<false>(p, q, sP, s_inj, s_plan, bid, n_fix);
     }
   }
   // every CTA read the counter before the first grid barrier
@@ -1317,9 +1326,10 @@ __global__ void __launch_bounds__(CK_THREADS, 2) check_pair_kernel(const __grid_
 
 // SPARE: some plan may have a spare parity to be verified on (two and more parities in the phase's code);
 // that pass needs a grid barrier, so only this instantiation is a cooperative launch.
+// s_plan: room for MAXN plans in shared memory.
 template <bool SPARE>
 __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, const float* sP, const unsigned long long* s_inj,
-                                         const unsigned bid, const unsigned gdim) {
+                                         CwPlan* s_plan, const unsigned bid, const unsigned gdim) {
   const Geom& g = p.g;
   const bool fwd = p.phase == CODENET_PHASE_FWD;
   const int B = p.B;
@@ -1327,6 +1337,14 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
   __shared__ unsigned s_res[MAXN];
   __shared__ unsigned s_final[MAXN];
   for (int t = tid; t < MAXN; t += CK_THREADS) s_res[t] = 0u;
+  // the plans, once per CTA, into shared memory: every element's decoding reads them, and from global memory each
+  // field would be one more round trip in front of the loads that depend on it
+  {
+    const uint32_t* from = reinterpret_cast<const uint32_t*>(p.plan);
+    uint32_t* to = reinterpret_cast<uint32_t*>(s_plan);
+    const int words = q.n_cw * (int)(sizeof(CwPlan) / sizeof(uint32_t));
+    for (int w = tid; w < words; w += CK_THREADS) to[w] = __ldcg(from + w);
+  }
   __syncthreads();
   const size_t gstride = (size_t)gdim * CK_THREADS;
   const size_t g0 = bid * (size_t)CK_THREADS + tid;
@@ -1337,7 +1355,7 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
     const size_t total = (size_t)q.n_cw * q.n_el;
     for (size_t idx = g0; idx < total; idx += gstride) {
       const int cw = (int)(idx / q.n_el);
-      const CwPlan& pl = p.plan[cw];
+      const CwPlan& pl = s_plan[cw];
       if (pl.state != 1 || pl.spare == 0u) continue;
       const size_t e = idx % q.n_el;
       const CwView yw = cw_view(p, q, s_inj, cw);
@@ -1359,7 +1377,7 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
   for (int cw = tid; cw < MAXN; cw += CK_THREADS) {
     unsigned st = 0u;
     if (cw < q.n_cw) {
-      const CwPlan& pl = p.plan[cw];
+      const CwPlan& pl = s_plan[cw];
       st = (unsigned)pl.state;
       if (SPARE && st == 1u && pl.spare != 0u && __uint_as_float(__ldcg(&p.st->resid[cw])) > pl.tau) st = 3u;
     }
@@ -1378,7 +1396,7 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
     if (tid < q.n_cw) {
       const unsigned long long data = q.kd >= 64 ? ~0ull : ((1ull << q.kd) - 1ull);
       unsigned long long mask = 0ull;
-      if (s_final[tid] == 1u) mask = p.plan[tid].F & data;
+      if (s_final[tid] == 1u) mask = s_plan[tid].F & data;
       else if (s_final[tid] == 3u && p.have_clean) mask = s_inj[tid] & data;
       s_touch[tid] = mask;
       if (mask) atomicOr(&s_nodes, mask);
@@ -1389,11 +1407,12 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
     const size_t per_node = (size_t)q.len * B;
     for (int node = 0; node < q.kd; ++node) {
       if (!((nodes >> node) & 1ull)) continue;
-      for (size_t idx = g0; idx < per_node; idx += gstride) {
-        const int b = (int)(idx % B), pos = (int)(idx / B);
+      // (32-bit index arithmetic: a node output has fewer than 2^32 elements, and 64-bit division is a long routine)
+      for (unsigned idx = (unsigned)g0; idx < (unsigned)per_node; idx += (unsigned)gstride) {
+        const int b = B == 1 ? 0 : (int)(idx % (unsigned)B), pos = B == 1 ? (int)idx : (int)(idx / (unsigned)B);
         const int gidx = node * q.len + pos;
         if (gidx >= nout) continue;
-        const float acc = sum_final_values(p, q, sP, s_inj, s_final, s_touch, node, idx);
+        const float acc = sum_final_values(p, q, sP, s_inj, s_final, s_touch, s_plan, node, idx);
         p.out[(size_t)b * nout + gidx] = finish_out(p, acc, (size_t)b * nout + gidx);
       }
     }
@@ -1406,7 +1425,7 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
       const size_t e = idx % q.n_el;
       float* yw = p.Yw + (size_t)cw * q.K * q.n_el;
       if (s_final[cw] == 1u) {
-        const CwPlan& pl = p.plan[cw];
+        const CwPlan& pl = s_plan[cw];
         float fix[MAXR];
         double par[MAXR];
         decode_at(cw_view(p, q, s_inj, cw), q, sP, pl, e, fix, par);
@@ -1422,7 +1441,8 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
       }
     }
   }
-  if (p.rep && bid == 0) {
+  // (without spare parities the plans are final as the check kernel's decision phase reported them)
+  if (SPARE && p.rep && bid == 0) {
     __shared__ float s_a[MAXN], s_b[MAXN];
     write_report(p, q.n_cw, s_final, s_a, s_b);
   }
@@ -1437,7 +1457,8 @@ __global__ void __launch_bounds__(CK_THREADS) fix_kernel(CheckParams p) {
   __shared__ unsigned long long s_inj[MAXN];
   for (int t = threadIdx.x; t < q.kd * q.r; t += CK_THREADS) sP[t] = q.P[t];
   build_hit_masks(p, q, s_inj);
-  fix_body<SPARE>(p, q, sP, s_inj, blockIdx.x, gridDim.x);
+  __shared__ CwPlan s_plan[MAXN];
+  fix_body<SPARE>(p, q, sP, s_inj, s_plan, blockIdx.x, gridDim.x);
 }
 
 // Soft errors in a node's own copy of its input sub-vector (the copy the activation / post-multiplication step
@@ -1770,3 +1791,4 @@ cudaError_t launch_sum_outputs(const Geom& g, int phase, int B, const float* Y, 
 }
 
 }  // namespace codenet
+
