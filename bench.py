@@ -297,9 +297,10 @@ def timed_steps(cn, torch, net, layers, cfg, wl, steps, warmup, inject, e2e=Fals
         # Recorded steps.  The K timed steps are cut into consecutive segments of 40 (and the rest), each one graph:
         # between two graph launches the device idles for 8-15 us, which a long recording makes rare.  40 is a
         # multiple of the input pool and of the staging ring, so one 40-step recording serves every whole segment.
-        # (Measured at K = 20: one recording of 20 steps, or any cut of them into 2-4 graphs with short ones first,
-        # all give 130.4-130.9 us per step against 125.0 at K = 1000: the first steps after the synchronisation
-        # that precedes the timed region run slower, however they are launched.)
+        # (A short run is not slower because it is short: the start of the timed region costs 12-13 us once.  What
+        # differs between windows of 10-20 steps is how many injected faults fall into them: the plan is fixed by
+        # seed and iteration, a step with a detected codeword takes 10-13 us longer, and iterations 5-24 of
+        # configuration 3 hold six of them where the long-run average is three.)
         it_ctr = torch.full((1,), warmup, dtype=torch.int32, device="cuda")
         faults = [cn.make_fault(seed=cfg.seed, layer=l, mode=mode, p=cfg.p, sigma=cfg.sigma, iteration_dev=it_ctr)
                   for l in range(L)]
