@@ -1352,22 +1352,23 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
   // phase V: residual of every decoding plan on its spare parities
   if (SPARE) {
     cg::grid_group grid = cg::this_grid();
-    const size_t total = (size_t)q.n_cw * q.n_el;
-    for (size_t idx = g0; idx < total; idx += gstride) {
-      const int cw = (int)(idx / q.n_el);
+    // only the codewords whose plan has a spare parity are walked (the others, nearly all, cost one test each)
+    for (int cw = 0; cw < q.n_cw; ++cw) {
       const CwPlan& pl = s_plan[cw];
       if (pl.state != 1 || pl.spare == 0u) continue;
-      const size_t e = idx % q.n_el;
       const CwView yw = cw_view(p, q, s_inj, cw);
-      float fix[MAXR];
-      double par[MAXR];
-      decode_at(yw, q, sP, pl, e, fix, par);
       float resid = 0.0f;
+      for (unsigned e = (unsigned)g0; e < (unsigned)q.n_el; e += (unsigned)gstride) {
+        float fix[MAXR];
+        double par[MAXR];
+        decode_at(yw, q, sP, pl, e, fix, par);
 #pragma unroll
-      for (int t = 0; t < MAXR; ++t)
-        if (t < q.r && ((pl.spare >> t) & 1u))
-          resid = fmaxf(resid, fabsf((float)(par[t] - (double)yw.at(q, q.kd + t, e))));
-      atomicMax(&s_res[cw], __float_as_uint(resid));
+        for (int t = 0; t < MAXR; ++t)
+          if (t < q.r && ((pl.spare >> t) & 1u))
+            resid = fmaxf(resid, fabsf((float)(par[t] - (double)yw.at(q, q.kd + t, e))));
+      }
+      resid = warp_max(resid);
+      if ((tid & 31) == 0 && resid > 0.0f) atomicMax(&s_res[cw], __float_as_uint(resid));
     }
     __syncthreads();
     for (int cw = tid; cw < q.n_cw; cw += CK_THREADS)
