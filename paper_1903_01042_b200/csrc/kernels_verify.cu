@@ -349,7 +349,7 @@ __device__ __forceinline__ void update_checksum_vectors(const CheckParams& p, co
   if (warp < first_warp) return;
   const int wpc = CK_WARPS - first_warp;
   const int gw = (gdim - 1 - bid) * wpc + (CK_WARPS - 1 - warp), nw = gdim * wpc;
-  const int n_uvec = g.M * g.Nn * g.ns, n_vvec = g.M * g.Nn * g.nsc;
+  const int n_uvec = g.M * g.Nn * g.ns;
   for (int vec = vec_begin + gw; vec < vec_end; vec += nw) {
     const bool is_u = vec < n_uvec;
     const int v2 = is_u ? vec : vec - n_uvec, nsl = is_u ? g.ns : g.nsc;
