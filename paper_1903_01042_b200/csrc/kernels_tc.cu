@@ -1,5 +1,5 @@
 // Tensor-core tiles for batches >= 64 (sm_100a): tcgen05.mma with accumulators in tensor memory,
-// operands staged in shared memory by TMA (cp.async.bulk.tensor, no multicast), an mbarrier ring
+// operands staged in shared memory by TMA (cp.async.bulk.tensor, every CTA loading its own tiles), an mbarrier ring
 // between a producer warp, an MMA warp and four epilogue warps.
 //
 // Forward node products (step O1):  Y[j][coded row][b] = sum_c W~[coded row][j*ldb + c] X[b][j*ldb + c]
