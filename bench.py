@@ -51,17 +51,32 @@ class ClockSampler(threading.Thread):
         self.sm_max = None
         self.source = None
         self.stop_flag = threading.Event()
+        # the library is opened here, before the timed region: a region of twenty steps lasts 2.5 ms, and a sampler
+        # that first has to load NVML inside it comes back with no sample at all
+        self.nv = self.handle = None
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            self.handle = nv.nvmlDeviceGetHandleByIndex(index)
+            self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(self.handle, nv.NVML_CLOCK_SM))
+            nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM)      # first calls are the slow ones
+            nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+            self.nv = nv
+        except Exception:
+            self.nv = None
 
     def _run_nvml(self):
-        import pynvml as nv
-        nv.nvmlInit()
-        h = nv.nvmlDeviceGetHandleByIndex(self.index)
-        self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+        nv, h = self.nv, self.handle
+        if nv is None:
+            raise RuntimeError("no NVML binding")
         self.source = "nvml"
+        n = 0
         while not self.stop_flag.is_set():
             self.sm.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
             self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
-            self.stop_flag.wait(self.period)
+            n += 1
+            # every half millisecond at first (short regions get a few samples), then at the set period
+            self.stop_flag.wait(0.0005 if n < 40 else self.period)
 
     def _run_smi(self):
         uuid = None
