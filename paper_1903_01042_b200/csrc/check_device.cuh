@@ -268,6 +268,10 @@ struct CwView {
   __device__ __forceinline__ float at(const PhaseGeom& q, int k, size_t e) const {
     return (((own >> k) & 1ull) ? yw : ys)[(size_t)k * q.n_el + e];
   }
+  // four consecutive elements (e a multiple of four; large batches: the buffers are 16-byte aligned)
+  __device__ __forceinline__ float4 at4(const PhaseGeom& q, int k, size_t e) const {
+    return *reinterpret_cast<const float4*>((((own >> k) & 1ull) ? yw : ys) + (size_t)k * q.n_el + e);
+  }
 };
 
 __device__ __forceinline__ bool lazy_copy(const CheckParams& p) {
@@ -344,6 +348,58 @@ __device__ __forceinline__ void decode_at(const CwView& yw, const PhaseGeom& q, 
       for (int t = 0; t < MAXR; ++t)
         if (t < q.r) par[t] += (double)sP[fda[a] * q.r + t] * (double)fix[a];
     }
+}
+
+// decode_at for a plan with ONE located data node and at most two parities, four consecutive elements at a time
+// (large batches): per element the same operations in the same order, with 16-byte loads and a quarter of the
+// instructions.  PAR: also re-encode the parities (for the verification on a spare one).
+template <bool PAR>
+__device__ __forceinline__ void decode1_at4(const CwView& yw, const PhaseGeom& q, const float* sP, const CwPlan& pl,
+                                            size_t e, float (&fix)[4], double (&par)[2][4]) {
+  const unsigned long long F = pl.F;
+  const int qa = pl.q[0], fd = pl.fd[0];
+  const float4 r4 = yw.at4(q, q.kd + qa, e);
+  double rhs[4] = {(double)r4.x, (double)r4.y, (double)r4.z, (double)r4.w};
+#pragma unroll
+  for (int t = 0; t < 2; ++t)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) par[t][c] = 0.0;
+#pragma unroll 1
+  for (int k0 = 0; k0 < q.kd; k0 += 8) {
+    float4 o8[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) o8[u] = yw.at4(q, min(k0 + u, q.kd - 1), e);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int k = k0 + u;
+      if (k >= q.kd || ((F >> k) & 1ull)) continue;
+      const double o[4] = {(double)o8[u].x, (double)o8[u].y, (double)o8[u].z, (double)o8[u].w};
+      const double pq = (double)sP[k * q.r + qa];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) rhs[c] -= pq * o[c];
+      if (PAR) {
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+          if (t < q.r) {
+            const double pt = (double)sP[k * q.r + t];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) par[t][c] += pt * o[c];
+          }
+      }
+    }
+  }
+  const double ainv = pl.ainv[0];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) fix[c] = (float)(ainv * rhs[c]);
+  if (PAR) {
+#pragma unroll
+    for (int t = 0; t < 2; ++t)
+      if (t < q.r) {
+        const double pt = (double)sP[fd * q.r + t];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) par[t][c] += pt * (double)fix[c];
+      }
+  }
 }
 
 // Report from the per-codeword plans; called by every thread of one CTA (>= 64 threads).
@@ -488,4 +544,39 @@ __device__ __forceinline__ float sum_final_values(const CheckParams& p, const Ph
       if (c0 + u < q.n_cw) acc += v[u];
   }
   return acc;
+}
+
+// sum_final_values for four consecutive elements of a large batch (e a multiple of four): 16-byte loads, eight
+// codewords in flight; a touched codeword whose plan has one located data node is decoded four elements at a time,
+// any other one element by element.  Per element the additions run in codeword order, as above.
+__device__ __forceinline__ void sum_final_values4(const CheckParams& p, const PhaseGeom& q, const float* sP,
+                                                  const unsigned long long* s_inj, const unsigned* s_final,
+                                                  const unsigned long long* s_touch, const CwPlan* plans, int node,
+                                                  size_t e, float (&acc)[4]) {
+#pragma unroll
+  for (int c = 0; c < 4; ++c) acc[c] = 0.0f;
+  for (int c0 = 0; c0 < q.n_cw; c0 += 8) {
+    float4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) v[u] = cw_view(p, q, s_inj, min(c0 + u, q.n_cw - 1)).at4(q, node, e);
+#pragma unroll 1
+    for (int cw = c0; cw < min(c0 + 8, q.n_cw); ++cw) {
+      if (!((s_touch[cw] >> node) & 1ull)) continue;
+      float d[4];
+      const CwPlan& pl = plans[cw];
+      if (s_final[cw] == 1u && pl.nfd == 1 && pl.fd[0] == node) {
+        double par[2][4];
+        decode1_at4<false>(cw_view(p, q, s_inj, cw), q, sP, pl, e, d, par);
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) d[c] = final_value(p, q, sP, s_inj, s_final, plans, cw, node, e + c);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (c0 + u == cw) v[u] = make_float4(d[0], d[1], d[2], d[3]);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      if (c0 + u < q.n_cw) { acc[0] += v[u].x; acc[1] += v[u].y; acc[2] += v[u].z; acc[3] += v[u].w; }
+  }
 }

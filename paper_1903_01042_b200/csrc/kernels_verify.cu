@@ -1358,14 +1358,30 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
       if (pl.state != 1 || pl.spare == 0u) continue;
       const CwView yw = cw_view(p, q, s_inj, cw);
       float resid = 0.0f;
-      for (unsigned e = (unsigned)g0; e < (unsigned)q.n_el; e += (unsigned)gstride) {
-        float fix[MAXR];
-        double par[MAXR];
-        decode_at(yw, q, sP, pl, e, fix, par);
+      if (lazy_copy(p) && pl.nfd == 1 && q.r <= 2) {
+        // large batches, one located data node: four batch entries per thread and round
+        for (unsigned e = (unsigned)g0 * 4u; e < (unsigned)q.n_el; e += (unsigned)gstride * 4u) {
+          float fix[4];
+          double par[2][4];
+          decode1_at4<true>(yw, q, sP, pl, e, fix, par);
 #pragma unroll
-        for (int t = 0; t < MAXR; ++t)
-          if (t < q.r && ((pl.spare >> t) & 1u))
-            resid = fmaxf(resid, fabsf((float)(par[t] - (double)yw.at(q, q.kd + t, e))));
+          for (int t = 0; t < 2; ++t)
+            if (t < q.r && ((pl.spare >> t) & 1u)) {
+              const float4 o = yw.at4(q, q.kd + t, e);
+              resid = fmaxf(resid, fmaxf(fmaxf(fabsf((float)(par[t][0] - (double)o.x)), fabsf((float)(par[t][1] - (double)o.y))),
+                                         fmaxf(fabsf((float)(par[t][2] - (double)o.z)), fabsf((float)(par[t][3] - (double)o.w)))));
+            }
+        }
+      } else {
+        for (unsigned e = (unsigned)g0; e < (unsigned)q.n_el; e += (unsigned)gstride) {
+          float fix[MAXR];
+          double par[MAXR];
+          decode_at(yw, q, sP, pl, e, fix, par);
+#pragma unroll
+          for (int t = 0; t < MAXR; ++t)
+            if (t < q.r && ((pl.spare >> t) & 1u))
+              resid = fmaxf(resid, fabsf((float)(par[t] - (double)yw.at(q, q.kd + t, e))));
+        }
       }
       resid = warp_max(resid);
       if ((tid & 31) == 0 && resid > 0.0f) atomicMax(&s_res[cw], __float_as_uint(resid));
@@ -1408,6 +1424,22 @@ __device__ __forceinline__ void fix_body(CheckParams& p, const PhaseGeom& q, con
     const size_t per_node = (size_t)q.len * B;
     for (int node = 0; node < q.kd; ++node) {
       if (!((nodes >> node) & 1ull)) continue;
+      if (lazy_copy(p)) {
+        // large batches (B a multiple of 32): four batch entries of one position per thread and round
+        for (unsigned idx = (unsigned)g0 * 4u; idx < (unsigned)per_node; idx += (unsigned)gstride * 4u) {
+          const int b = (int)(idx % (unsigned)B), pos = (int)(idx / (unsigned)B);
+          const int gidx = node * q.len + pos;
+          if (gidx >= nout) continue;
+          float acc[4];
+          sum_final_values4(p, q, sP, s_inj, s_final, s_touch, s_plan, node, idx, acc);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const size_t oi = (size_t)(b + c) * nout + gidx;
+            p.out[oi] = finish_out(p, acc[c], oi);
+          }
+        }
+        continue;
+      }
       // (32-bit index arithmetic: a node output has fewer than 2^32 elements, and 64-bit division is a long routine)
       for (unsigned idx = (unsigned)g0; idx < (unsigned)per_node; idx += (unsigned)gstride) {
         const int b = B == 1 ? 0 : (int)(idx % (unsigned)B), pos = B == 1 ? (int)idx : (int)(idx / (unsigned)B);
