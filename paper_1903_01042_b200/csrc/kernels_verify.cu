@@ -1256,7 +1256,8 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
                                : state == 3 ? (uint32_t)(p.have_clean ? CODENET_FALLBACK : CODENET_FAILED)
                                : state == 4 ? (uint32_t)CODENET_DISAGREE
                                             : (uint32_t)CODENET_CLEAN;
-        if (outcome != CODENET_CLEAN) atomicMax(&r->status, outcome);
+        // (a wait that ran out in a tensor-core kernel outranks every outcome: the status was set to TIMEOUT above)
+        if (outcome != CODENET_CLEAN && !(p.tc_flag && *p.tc_flag)) atomicMax(&r->status, outcome);
         atomicMin(reinterpret_cast<unsigned*>(&r->min_margin_hit), __float_as_uint(cw_min_hit));
         atomicMax(reinterpret_cast<unsigned*>(&r->max_margin_clean), __float_as_uint(cw_max_clean));
       }
