@@ -1242,6 +1242,16 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
         }
       }
       pl.state = state;
+      if (p.inline_fix || p.tail_fix) {
+        // one counter tells the waiting CTAs both things: how many codewords have decided (low half) and how many of
+        // them need work (high half)
+        __threadfence();
+        atomicAdd(&p.st->done_d, 1u + (state != 0 ? 0x10000u : 0u));
+      } else if (state != 0) {
+        atomicOr(&p.st->need_fix, 1u);   // read by the fix kernel that follows
+      }
+      // the report after the counter: the CTAs that wait for the counter read the plans, not the report, and the fence
+      // in front of it then has the plan's stores alone to wait for
       if (p.rep != nullptr) {
         codenet_report_t* r = p.rep;
         r->flagged_mask[cw] = detected ? F : 0ull;
@@ -1260,14 +1270,6 @@ __device__ __forceinline__ void check_body(CheckParams& p, const unsigned bid, c
         if (outcome != CODENET_CLEAN && !(p.tc_flag && *p.tc_flag)) atomicMax(&r->status, outcome);
         atomicMin(reinterpret_cast<unsigned*>(&r->min_margin_hit), __float_as_uint(cw_min_hit));
         atomicMax(reinterpret_cast<unsigned*>(&r->max_margin_clean), __float_as_uint(cw_max_clean));
-      }
-      if (p.inline_fix || p.tail_fix) {
-        // one counter tells the waiting CTAs both things: how many codewords have decided (low half) and how many of
-        // them need work (high half)
-        __threadfence();
-        atomicAdd(&p.st->done_d, 1u + (state != 0 ? 0x10000u : 0u));
-      } else if (state != 0) {
-        atomicOr(&p.st->need_fix, 1u);   // read by the fix kernel that follows
       }
     }
     __syncthreads();
